@@ -1,0 +1,122 @@
+/*
+ * cubicquant.h -- C ABI of the B200 (sm_100a) CubicQuant packed-weight GEMV / GEMM library.
+ *
+ * The library computes   y[M,N] = x[M,K] * What[N,K]^T   directly from packed B-bit
+ * (1..8) weight codes whose per-group reconstruction levels follow the paper's monotone
+ * cubic (Section 2.2, Eq. cubic), in two activation modes (Section 5.3 model dtype,
+ * Section 5.4 Dynamic A8).
+ *
+ * Conventions common to every call
+ *   - All pointers are DEVICE pointers unless the name says "host".  The caller owns every
+ *     buffer; the library allocates no device memory and never synchronises the device
+ *     (except cq_gemm_host, which waits for its own copies).
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *   - Return value: CQ_OK or a negative CQ_ERR_* code.  Argument errors are found on the
+ *     host before anything is launched.
+ *   - Logical weight matrix: N output channels x K input channels; groups are runs of G
+ *     consecutive input channels inside one output row (Section 2.3).
+ *   - Canonical (interchange) format, the paper's packed checkpoint view:
+ *       codes  uint8 [N][ceil(K*B/8)]  continuous LSB-first bitstream per row, field j at bit
+ *                                      j*B (Eq. gpu-packed-extraction); B-bit two's complement,
+ *                                      pattern -2^(B-1) reserved and decoding to 0 (Eq. codes);
+ *                                      W1: bit 1 = +1, bit 0 = -1.
+ *       scale  float  [N][K/G]         s >= 0 (FP32, Appendix A item 3)
+ *       a, b   fp16   [N][K/G]         shape coefficients as IEEE binary16 bit patterns
+ *   - Device layout: private, tiled and interleaved for 128-bit coalesced loads with the
+ *     group parameters stored beside the codes of their tile; produced by cq_repack and
+ *     inverted bit-exactly by cq_unpack.
+ *   - Supported: B in 1..8; G in {32, 64, 128}; K % G == 0; M, N, K >= 1.  K and N need not be
+ *     multiples of the 128 x 128 tile (the layout pads).
+ */
+#ifndef CUBICQUANT_H_
+#define CUBICQUANT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    CQ_OK = 0,
+    CQ_ERR_INVALID_ARG = -1, /* null pointer, M/N/K <= 0, B outside 1..8, unknown mode */
+    CQ_ERR_UNSUPPORTED = -2, /* K % G != 0, G not in {32,64,128} */
+    CQ_ERR_ALIGNMENT = -3,   /* a pointer is not 16-byte aligned */
+    CQ_ERR_WORKSPACE = -4,   /* workspace_bytes smaller than cq_workspace_bytes() */
+    CQ_ERR_ARCH = -5,        /* current device is not compute capability 10.x */
+    CQ_ERR_CUDA = -6,        /* a CUDA runtime call or launch failed; see cq_last_cuda_error() */
+    CQ_ERR_TIMEOUT = -7      /* a bounded device-side wait gave up (reported by cq_gemm_status) */
+};
+
+enum { CQ_MODEL_DTYPE = 0, CQ_DYN_A8 = 1 };
+
+/* Human-readable name of a status code (static string). */
+const char *cq_status_string(int status);
+/* cudaError_t value of the last failed CUDA call made by this library on this thread (0 if none). */
+int cq_last_cuda_error(void);
+
+/* Bytes of the canonical code tensor: N * ceil(K*B/8). */
+size_t cq_canonical_code_bytes(int B, int64_t N, int64_t K);
+/* Effective stored bits per weight of the canonical format, B + 64/G (Eq. effective-bits). */
+double cq_effective_bits(int B, int G);
+/* Bytes of the device layout for an N x K matrix (codes + co-located parameters, including the
+ * padding of N and K up to multiples of 128).  0 if the arguments are unsupported. */
+size_t cq_layout_bytes(int B, int G, int64_t N, int64_t K);
+/* Bytes of scratch cq_gemm needs for this problem (split-K partial sums and arrival counters;
+ * Dynamic A8 adds the INT8 activation carrier and its row scales).  Never 0 for valid input. */
+size_t cq_workspace_bytes(int B, int G, int64_t M, int64_t N, int64_t K, int mode);
+/* Zero the arrival counters of a workspace.  Call once after allocating it (and after any
+ * cq_gemm that returned an error); cq_gemm leaves the counters zero when it completes. */
+int cq_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
+
+/* Signed logical codes k[N][K] (int8; W1: +-1) -> canonical packed bitstream (Section 2.1,
+ * Eq. gpu-packed-extraction read backwards).  `codes` must hold cq_canonical_code_bytes(). */
+int cq_pack_codes(const int8_t *k, int B, int64_t N, int64_t K, uint8_t *codes, void *stream);
+
+/* Canonical format -> device layout (Section 2.1/2.3 data, re-tiled; a bijection). */
+int cq_repack(const uint8_t *codes, const float *scale, const uint16_t *a, const uint16_t *b, int B, int G, int64_t N,
+              int64_t K, void *layout, void *stream);
+/* Device layout -> canonical format; returns exactly the bytes given to cq_repack. */
+int cq_unpack(const void *layout, int B, int G, int64_t N, int64_t K, uint8_t *codes, float *scale, uint16_t *a,
+              uint16_t *b, void *stream);
+
+/* The hot path.  y[M][N] (bf16 bits, row-major) = x[M][K] (bf16 bits, row-major) * What^T.
+ *   mode CQ_MODEL_DTYPE: continuous reconstruction of Eq. cubic; fp32 accumulation (Section 5.3).
+ *   mode CQ_DYN_A8:      per-row absmax INT8 activations (Eq. a8-activation-scale/-quantization),
+ *                        INT8 weight carriers (Eq. carrier), int32 group partials, fp32 rescale
+ *                        (Eq. a8-output).
+ * M <= 16 runs the split-K tensor-core GEMV; larger M the tcgen05/TMEM GEMM.
+ * x, y, layout and workspace must be 16-byte aligned; x and y must not alias. */
+int cq_gemm(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, int64_t M, int64_t N, int64_t K,
+            int mode, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Same product with HOST activations and HOST output: copies x_host to the device, runs cq_gemm
+ * and copies y back, all on `stream`, then waits for the stream.  x_dev (M*K bf16) and y_dev
+ * (M*N bf16) are caller-provided device staging buffers.  Pinned host memory makes the copies
+ * asynchronous; pageable memory also works. */
+int cq_gemm_host(const void *layout, int B, int G, const uint16_t *x_host, uint16_t *y_host, uint16_t *x_dev,
+                 uint16_t *y_dev, int64_t M, int64_t N, int64_t K, int mode, void *workspace, size_t workspace_bytes,
+                 void *stream);
+
+/* Pieces of the path exposed for parity tests. */
+
+/* Dynamic-A8 activation quantiser (Eq. a8-activation-scale, Eq. a8-activation-quantization):
+ * x8[M][K] int8 and dx[M] float from x[M][K] bf16.  fp32 arithmetic: xbar = max(max|x|, 1e-10f),
+ * dx = xbar / 127 (IEEE division), x8 = clip(round-half-away(x / dx), -127, 127). */
+int cq_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, float *dx, void *stream);
+/* Non-negative reconstruction levels of every group (Appendix B): levels[N][K/G][L] float,
+ * L = 2^(B-1) (W1: L = 1, the scale). */
+int cq_decode_levels(const void *layout, int B, int G, int64_t N, int64_t K, float *levels, void *stream);
+/* Non-negative INT8 carriers of every group (Eq. carrier): carriers[N][K/G][L] int8. */
+int cq_decode_carriers(const void *layout, int B, int G, int64_t N, int64_t K, int8_t *carriers, void *stream);
+/* Dense reconstruction What[N][K] float (sign * level of every code; reserved pattern -> 0). */
+int cq_decode_weights(const void *layout, int B, int G, int64_t N, int64_t K, float *What, void *stream);
+/* Integer group partials of Eq. a8-output: P[M][N][K/G] int32 from x8[M][K]. */
+int cq_debug_a8_partials(const void *layout, int B, int G, const int8_t *x8, int64_t M, int64_t N, int64_t K,
+                         int32_t *P, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CUBICQUANT_H_ */

@@ -1,0 +1,208 @@
+"""ctypes binding of the C ABI (include/cubicquant.h).  Argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libcubicquant.so")
+
+CQ_MODEL_DTYPE = 0
+CQ_DYN_A8 = 1
+
+_lib = None
+
+
+class CubicQuantError(RuntimeError):
+    pass
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def lib():
+    """The loaded shared library.  Fails loudly when it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise CubicQuantError(f"{_LIB_PATH} is missing: build it with `python -m paper_2608_06763_b200.build` "
+                                  "(there is no fallback path)")
+        L = C.CDLL(_LIB_PATH)
+        vp, i, i64, sz = C.c_void_p, C.c_int, C.c_int64, C.c_size_t
+        L.cq_status_string.restype = C.c_char_p
+        L.cq_status_string.argtypes = [i]
+        L.cq_last_cuda_error.restype = i
+        L.cq_canonical_code_bytes.restype = sz
+        L.cq_canonical_code_bytes.argtypes = [i, i64, i64]
+        L.cq_effective_bits.restype = C.c_double
+        L.cq_effective_bits.argtypes = [i, i]
+        L.cq_layout_bytes.restype = sz
+        L.cq_layout_bytes.argtypes = [i, i, i64, i64]
+        L.cq_workspace_bytes.restype = sz
+        L.cq_workspace_bytes.argtypes = [i, i, i64, i64, i64, i]
+        L.cq_workspace_init.argtypes = [vp, sz, vp]
+        L.cq_pack_codes.argtypes = [vp, i, i64, i64, vp, vp]
+        L.cq_repack.argtypes = [vp, vp, vp, vp, i, i, i64, i64, vp, vp]
+        L.cq_unpack.argtypes = [vp, i, i, i64, i64, vp, vp, vp, vp, vp]
+        L.cq_gemm.argtypes = [vp, i, i, vp, vp, i64, i64, i64, i, vp, sz, vp]
+        L.cq_gemm_host.argtypes = [vp, i, i, vp, vp, vp, vp, i64, i64, i64, i, vp, sz, vp]
+        L.cq_quantize_a8.argtypes = [vp, i64, i64, vp, vp, vp]
+        L.cq_decode_levels.argtypes = [vp, i, i, i64, i64, vp, vp]
+        L.cq_decode_carriers.argtypes = [vp, i, i, i64, i64, vp, vp]
+        L.cq_decode_weights.argtypes = [vp, i, i, i64, i64, vp, vp]
+        L.cq_debug_a8_partials.argtypes = [vp, i, i, vp, i64, i64, i64, vp, vp]
+        for name in ("cq_workspace_init", "cq_pack_codes", "cq_repack", "cq_unpack", "cq_gemm", "cq_gemm_host",
+                     "cq_quantize_a8", "cq_decode_levels", "cq_decode_carriers", "cq_decode_weights",
+                     "cq_debug_a8_partials"):
+            getattr(L, name).restype = i
+        _lib = L
+    return _lib
+
+
+def _check(status: int, what: str):
+    if status != 0:
+        L = lib()
+        raise CubicQuantError(f"{what}: {L.cq_status_string(status).decode()} (cuda error {L.cq_last_cuda_error()})")
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t: torch.Tensor) -> int:
+    assert t.is_cuda and t.is_contiguous(), "device, contiguous tensors only"
+    return t.data_ptr()
+
+
+def cq_status_string(status: int) -> str:
+    return lib().cq_status_string(status).decode()
+
+
+def cq_canonical_code_bytes(B, N, K) -> int:
+    return lib().cq_canonical_code_bytes(B, N, K)
+
+
+def cq_effective_bits(B, G) -> float:
+    return lib().cq_effective_bits(B, G)
+
+
+def cq_layout_bytes(B, G, N, K) -> int:
+    return lib().cq_layout_bytes(B, G, N, K)
+
+
+def cq_workspace_bytes(B, G, M, N, K, mode) -> int:
+    return lib().cq_workspace_bytes(B, G, M, N, K, mode)
+
+
+def cq_workspace_init(workspace: torch.Tensor):
+    _check(lib().cq_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
+           "cq_workspace_init")
+
+
+def cq_pack_codes(k: torch.Tensor, B: int) -> torch.Tensor:
+    """int8 logical codes [N, K] -> canonical packed bytes [N, ceil(K*B/8)] (uint8, device)."""
+    N, K = k.shape
+    out = torch.empty((N, (K * B + 7) // 8), dtype=torch.uint8, device=k.device)
+    _check(lib().cq_pack_codes(_ptr(k), B, N, K, _ptr(out), _stream()), "cq_pack_codes")
+    return out
+
+
+@dataclass
+class PackedWeights:
+    """A matrix in the device layout (owned torch buffer plus its format)."""
+    layout: torch.Tensor
+    B: int
+    G: int
+    N: int
+    K: int
+
+
+def cq_repack(codes, scale, a, b, B, G, N, K) -> PackedWeights:
+    """Canonical tensors (device: codes uint8, scale fp32, a/b fp16) -> device layout."""
+    nbytes = cq_layout_bytes(B, G, N, K)
+    if nbytes == 0:
+        _check(lib().cq_repack(0, 0, 0, 0, B, G, N, K, 0, 0) or -2, "cq_repack")
+    layout = torch.empty(nbytes, dtype=torch.uint8, device=codes.device)
+    _check(lib().cq_repack(_ptr(codes), _ptr(scale), _ptr(a), _ptr(b), B, G, N, K, _ptr(layout), _stream()),
+           "cq_repack")
+    return PackedWeights(layout, B, G, N, K)
+
+
+def cq_unpack(pw: PackedWeights):
+    dev = pw.layout.device
+    codes = torch.empty((pw.N, (pw.K * pw.B + 7) // 8), dtype=torch.uint8, device=dev)
+    ng = pw.K // pw.G
+    scale = torch.empty((pw.N, ng), dtype=torch.float32, device=dev)
+    a = torch.empty((pw.N, ng), dtype=torch.float16, device=dev)
+    b = torch.empty((pw.N, ng), dtype=torch.float16, device=dev)
+    _check(lib().cq_unpack(_ptr(pw.layout), pw.B, pw.G, pw.N, pw.K, _ptr(codes), _ptr(scale), _ptr(a), _ptr(b),
+                           _stream()), "cq_unpack")
+    return codes, scale, a, b
+
+
+def cq_gemm(pw: PackedWeights, x: torch.Tensor, mode: int = CQ_MODEL_DTYPE, workspace: torch.Tensor | None = None,
+            out: torch.Tensor | None = None) -> torch.Tensor:
+    """y[M, N] bf16 = x[M, K] bf16 * What^T from the packed weights."""
+    assert x.dtype == torch.bfloat16 and x.dim() == 2 and x.shape[1] == pw.K
+    M = x.shape[0]
+    if workspace is None:
+        workspace = torch.zeros(cq_workspace_bytes(pw.B, pw.G, M, pw.N, pw.K, mode), dtype=torch.uint8, device=x.device)
+    y = out if out is not None else torch.empty((M, pw.N), dtype=torch.bfloat16, device=x.device)
+    _check(lib().cq_gemm(_ptr(pw.layout), pw.B, pw.G, _ptr(x), _ptr(y), M, pw.N, pw.K, mode, _ptr(workspace),
+                         workspace.numel(), _stream()), "cq_gemm")
+    return y
+
+
+def cq_gemm_host(pw: PackedWeights, x_host: torch.Tensor, y_host: torch.Tensor, x_dev: torch.Tensor,
+                 y_dev: torch.Tensor, mode: int, workspace: torch.Tensor):
+    """Host-buffer variant: copies x in, runs the product, copies y out, waits."""
+    M = x_host.shape[0]
+    assert not x_host.is_cuda and not y_host.is_cuda
+    _check(lib().cq_gemm_host(_ptr(pw.layout), pw.B, pw.G, x_host.data_ptr(), y_host.data_ptr(), _ptr(x_dev),
+                              _ptr(y_dev), M, pw.N, pw.K, mode, _ptr(workspace), workspace.numel(), _stream()),
+           "cq_gemm_host")
+    return y_host
+
+
+def cq_quantize_a8(x: torch.Tensor):
+    M, K = x.shape
+    x8 = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    dx = torch.empty(M, dtype=torch.float32, device=x.device)
+    _check(lib().cq_quantize_a8(_ptr(x), M, K, _ptr(x8), _ptr(dx), _stream()), "cq_quantize_a8")
+    return x8, dx
+
+
+def _num_levels(B):
+    return 1 if B == 1 else 1 << (B - 1)
+
+
+def cq_decode_levels(pw: PackedWeights) -> torch.Tensor:
+    out = torch.empty((pw.N, pw.K // pw.G, _num_levels(pw.B)), dtype=torch.float32, device=pw.layout.device)
+    _check(lib().cq_decode_levels(_ptr(pw.layout), pw.B, pw.G, pw.N, pw.K, _ptr(out), _stream()), "cq_decode_levels")
+    return out
+
+
+def cq_decode_carriers(pw: PackedWeights) -> torch.Tensor:
+    out = torch.empty((pw.N, pw.K // pw.G, _num_levels(pw.B)), dtype=torch.int8, device=pw.layout.device)
+    _check(lib().cq_decode_carriers(_ptr(pw.layout), pw.B, pw.G, pw.N, pw.K, _ptr(out), _stream()),
+           "cq_decode_carriers")
+    return out
+
+
+def cq_decode_weights(pw: PackedWeights) -> torch.Tensor:
+    out = torch.empty((pw.N, pw.K), dtype=torch.float32, device=pw.layout.device)
+    _check(lib().cq_decode_weights(_ptr(pw.layout), pw.B, pw.G, pw.N, pw.K, _ptr(out), _stream()),
+           "cq_decode_weights")
+    return out
+
+
+def cq_debug_a8_partials(pw: PackedWeights, x8: torch.Tensor) -> torch.Tensor:
+    M = x8.shape[0]
+    out = torch.empty((M, pw.N, pw.K // pw.G), dtype=torch.int32, device=x8.device)
+    _check(lib().cq_debug_a8_partials(_ptr(pw.layout), pw.B, pw.G, _ptr(x8), M, pw.N, pw.K, _ptr(out), _stream()),
+           "cq_debug_a8_partials")
+    return out

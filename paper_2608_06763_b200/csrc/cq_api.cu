@@ -1,0 +1,213 @@
+// C ABI of the library (include/cubicquant.h): argument validation on the host, then launches.
+#include "../../include/cubicquant.h"
+
+#include <cuda_runtime.h>
+
+#include "cq_common.cuh"
+#include "cq_internal.h"
+
+namespace cq {
+
+static thread_local int g_last_cuda_error = 0;
+
+int gemv_split_k(const Dims &d);
+int gemm_tc_available();
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+Workspace plan_workspace(const Dims &d, int64_t M, int mode) {
+    Workspace w{};
+    const int64_t Np = (int64_t)d.NB * TILE, Kp = (int64_t)d.KT * TILE;
+    const int64_t Mc = M < 16 ? M : 16;  // rows handled by one small-M launch
+    w.split_k = gemv_split_k(d);
+    size_t off = 0;
+    w.counters_off = off; w.counters_bytes = align_up((size_t)d.NB * 4, 256); off += w.counters_bytes;
+    w.status_off = off; off += 256;
+    w.partial_off = off; w.partial_bytes = align_up((size_t)w.split_k * Mc * Np * 4, 256); off += w.partial_bytes;
+    if (mode == CQ_DYN_A8) {
+        w.x8_off = off; w.x8_bytes = align_up((size_t)(M + 127) / 128 * 128 * Kp, 256); off += w.x8_bytes;
+        w.dx_off = off; w.dx_bytes = align_up((size_t)M * 4, 256); off += w.dx_bytes;
+    }
+    w.total = off;
+    return w;
+}
+
+static int check_format(int B, int G, int64_t N, int64_t K) {
+    if (B < 1 || B > 8 || N <= 0 || K <= 0 || G <= 0) return CQ_ERR_INVALID_ARG;
+    if (G != 32 && G != 64 && G != 128) return CQ_ERR_UNSUPPORTED;
+    if (K % G != 0) return CQ_ERR_UNSUPPORTED;
+    return CQ_OK;
+}
+static bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+static int check_arch() {
+    static thread_local int cached_dev = -1, cached_ok = 0;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { g_last_cuda_error = (int)e; return CQ_ERR_CUDA; }
+    if (dev != cached_dev) {
+        int major = 0;
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return CQ_ERR_CUDA; }
+        cached_dev = dev;
+        cached_ok = (major == 10);
+    }
+    return cached_ok ? CQ_OK : CQ_ERR_ARCH;
+}
+
+static int wrap(cudaError_t e) {
+    if (e == cudaSuccess) return CQ_OK;
+    g_last_cuda_error = (int)e;
+    return CQ_ERR_CUDA;
+}
+
+}  // namespace cq
+
+using namespace cq;
+
+#pragma GCC visibility push(default)
+extern "C" {
+
+const char *cq_status_string(int status) {
+    switch (status) {
+        case CQ_OK: return "CQ_OK";
+        case CQ_ERR_INVALID_ARG: return "CQ_ERR_INVALID_ARG";
+        case CQ_ERR_UNSUPPORTED: return "CQ_ERR_UNSUPPORTED";
+        case CQ_ERR_ALIGNMENT: return "CQ_ERR_ALIGNMENT";
+        case CQ_ERR_WORKSPACE: return "CQ_ERR_WORKSPACE";
+        case CQ_ERR_ARCH: return "CQ_ERR_ARCH";
+        case CQ_ERR_CUDA: return "CQ_ERR_CUDA";
+        case CQ_ERR_TIMEOUT: return "CQ_ERR_TIMEOUT";
+        default: return "CQ_ERR_UNKNOWN";
+    }
+}
+
+int cq_last_cuda_error(void) { return g_last_cuda_error; }
+
+size_t cq_canonical_code_bytes(int B, int64_t N, int64_t K) {
+    if (B < 1 || B > 8 || N <= 0 || K <= 0) return 0;
+    return (size_t)N * (size_t)((K * B + 7) / 8);
+}
+
+double cq_effective_bits(int B, int G) { return (double)B + 64.0 / (double)G; }
+
+size_t cq_layout_bytes(int B, int G, int64_t N, int64_t K) {
+    if (check_format(B, G, N, K) != CQ_OK) return 0;
+    const Dims d = make_dims(B, G, N, K);
+    return (size_t)d.NB * d.KT * (size_t)d.tile_bytes;
+}
+
+size_t cq_workspace_bytes(int B, int G, int64_t M, int64_t N, int64_t K, int mode) {
+    if (check_format(B, G, N, K) != CQ_OK || M <= 0 || (mode != CQ_MODEL_DTYPE && mode != CQ_DYN_A8)) return 0;
+    return plan_workspace(make_dims(B, G, N, K), M, mode).total;
+}
+
+int cq_workspace_init(void *workspace, size_t workspace_bytes, void *stream) {
+    if (!workspace || workspace_bytes == 0) return CQ_ERR_INVALID_ARG;
+    // counters and the status word sit at the front of the workspace; zeroing everything is simplest
+    return wrap(cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream));
+}
+
+int cq_pack_codes(const int8_t *k, int B, int64_t N, int64_t K, uint8_t *codes, void *stream) {
+    if (!k || !codes || B < 1 || B > 8 || N <= 0 || K <= 0) return CQ_ERR_INVALID_ARG;
+    return wrap(launch_pack_codes(k, B, N, K, codes, (cudaStream_t)stream));
+}
+
+int cq_repack(const uint8_t *codes, const float *scale, const uint16_t *a, const uint16_t *b, int B, int G, int64_t N,
+              int64_t K, void *layout, void *stream) {
+    if (!codes || !scale || !a || !b || !layout) return CQ_ERR_INVALID_ARG;
+    int st = check_format(B, G, N, K);
+    if (st != CQ_OK) return st;
+    if (misaligned(layout)) return CQ_ERR_ALIGNMENT;
+    return wrap(launch_repack(codes, scale, a, b, make_dims(B, G, N, K), layout, (cudaStream_t)stream));
+}
+
+int cq_unpack(const void *layout, int B, int G, int64_t N, int64_t K, uint8_t *codes, float *scale, uint16_t *a,
+              uint16_t *b, void *stream) {
+    if (!codes || !scale || !a || !b || !layout) return CQ_ERR_INVALID_ARG;
+    int st = check_format(B, G, N, K);
+    if (st != CQ_OK) return st;
+    if (misaligned(layout)) return CQ_ERR_ALIGNMENT;
+    return wrap(launch_unpack(layout, make_dims(B, G, N, K), codes, scale, a, b, (cudaStream_t)stream));
+}
+
+int cq_gemm(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, int64_t M, int64_t N, int64_t K,
+            int mode, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!layout || !x || !y || !workspace || M <= 0) return CQ_ERR_INVALID_ARG;
+    if (mode != CQ_MODEL_DTYPE && mode != CQ_DYN_A8) return CQ_ERR_INVALID_ARG;
+    int st = check_format(B, G, N, K);
+    if (st != CQ_OK) return st;
+    if (misaligned(layout) || misaligned(x) || misaligned(y) || misaligned(workspace)) return CQ_ERR_ALIGNMENT;
+    const Dims d = make_dims(B, G, N, K);
+    const Workspace plan = plan_workspace(d, M, mode);
+    if (workspace_bytes < plan.total) return CQ_ERR_WORKSPACE;
+    st = check_arch();
+    if (st != CQ_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    uint8_t *ws = (uint8_t *)workspace;
+    if (M <= 16) return wrap(launch_gemv(layout, d, x, y, M, mode, ws, plan, s));
+    if (gemm_tc_available()) return wrap(launch_gemm_tc(layout, d, x, y, M, mode, ws, plan, s));
+    // conservative route: 16 rows at a time through the small-M kernel (weights re-streamed per chunk)
+    for (int64_t m0 = 0; m0 < M; m0 += 16) {
+        const int64_t mc = (M - m0 < 16) ? (M - m0) : 16;
+        cudaError_t e = launch_gemv(layout, d, x + m0 * K, y + m0 * N, mc, mode, ws, plan, s);
+        if (e != cudaSuccess) return wrap(e);
+    }
+    return CQ_OK;
+}
+
+int cq_gemm_host(const void *layout, int B, int G, const uint16_t *x_host, uint16_t *y_host, uint16_t *x_dev,
+                 uint16_t *y_dev, int64_t M, int64_t N, int64_t K, int mode, void *workspace, size_t workspace_bytes,
+                 void *stream) {
+    if (!x_host || !y_host || !x_dev || !y_dev || M <= 0 || N <= 0 || K <= 0) return CQ_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return wrap(e);
+    int st = cq_gemm(layout, B, G, x_dev, y_dev, M, N, K, mode, workspace, workspace_bytes, stream);
+    if (st != CQ_OK) return st;
+    e = cudaMemcpyAsync(y_host, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return wrap(e);
+    return wrap(cudaStreamSynchronize(s));
+}
+
+int cq_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, float *dx, void *stream) {
+    if (!x || !x8 || !dx || M <= 0 || K <= 0) return CQ_ERR_INVALID_ARG;
+    return wrap(launch_quantize_a8(x, M, K, x8, K, dx, (cudaStream_t)stream));
+}
+
+#define CQ_DEBUG_PROLOGUE()                                   \
+    if (!layout) return CQ_ERR_INVALID_ARG;                   \
+    {                                                         \
+        int st_ = check_format(B, G, N, K);                   \
+        if (st_ != CQ_OK) return st_;                         \
+    }                                                         \
+    if (misaligned(layout)) return CQ_ERR_ALIGNMENT;          \
+    const Dims d = make_dims(B, G, N, K);
+
+int cq_decode_levels(const void *layout, int B, int G, int64_t N, int64_t K, float *levels, void *stream) {
+    if (!levels) return CQ_ERR_INVALID_ARG;
+    CQ_DEBUG_PROLOGUE();
+    return wrap(launch_decode_levels(layout, d, levels, (cudaStream_t)stream));
+}
+
+int cq_decode_carriers(const void *layout, int B, int G, int64_t N, int64_t K, int8_t *carriers, void *stream) {
+    if (!carriers) return CQ_ERR_INVALID_ARG;
+    CQ_DEBUG_PROLOGUE();
+    return wrap(launch_decode_carriers(layout, d, carriers, (cudaStream_t)stream));
+}
+
+int cq_decode_weights(const void *layout, int B, int G, int64_t N, int64_t K, float *What, void *stream) {
+    if (!What) return CQ_ERR_INVALID_ARG;
+    CQ_DEBUG_PROLOGUE();
+    return wrap(launch_decode_weights(layout, d, What, (cudaStream_t)stream));
+}
+
+int cq_debug_a8_partials(const void *layout, int B, int G, const int8_t *x8, int64_t M, int64_t N, int64_t K,
+                         int32_t *P, void *stream) {
+    if (!x8 || !P || M <= 0) return CQ_ERR_INVALID_ARG;
+    CQ_DEBUG_PROLOGUE();
+    return wrap(launch_a8_partials(layout, d, x8, M, P, (cudaStream_t)stream));
+}
+
+}  // extern "C"
+#pragma GCC visibility pop

@@ -1,0 +1,148 @@
+// Shared definitions of the CubicQuant sm_100a library: the private device layout and the
+// bit-field extraction every kernel uses.
+//
+// Device layout (what cq_repack writes; Section 2.1 / 2.3 data re-tiled, a bijection):
+//
+//   The N x K code matrix is padded to Np x Kp (multiples of 128) and cut into 128 x 128 tiles,
+//   stored tile after tile with the K index fastest: tile (nb, kb) at (nb * KT + kb) * tile_bytes.
+//   A tile is   [codes: 8 row blocks of 16 rows x 128 k][params: 128 rows x (128/G) groups x 8 B].
+//   The 8-byte parameter record of a (row, group) is {float s, half a, half b}; the sign bit of s
+//   (s >= 0 in the format) flags a group that contains the reserved code pattern.
+//
+//   Inside a row block, lane l = 4*g + t of a warp owns rows {g, g+8} and, for each of the eight
+//   16-wide k chunks j, the four k positions 16 j + 4 t + {0,1,2,3}: exactly the A fragment of a
+//   warp-level m16n8k16 MMA (and, two chunks at a time, of the m16n8k32 INT8 MMA).  Its 64 codes
+//   form 32 pairs p = 4 j + i, register i = {row g | k+0,1}, {row g+8 | k+0,1}, {row g | k+2,3},
+//   {row g+8 | k+2,3}; a pair sits in one 32-bit word with its first code in the low and its
+//   second code in the high 16 bits, so both are extracted by one mask.
+//
+//   Stored code u = k + 2^(B-1) (offset binary; u = 0 is the reserved pattern), W1: u = bit.
+//   u is split into bit planes of power-of-two width (B = 3 -> 2+1, 5 -> 4+1, 6 -> 4+2,
+//   7 -> 4+2+1) so every field is extracted with shifts and masks only.  A plane of width pw puts
+//   pair p in word p / (16/pw) at bit (p % (16/pw)) * pw.  A lane's 2B words are stored as
+//   16-byte quads, quad Q of lane l at ((Q * 32) + l) * 16 inside the row block (then an 8-byte
+//   tail when 2B is not a multiple of 4), so every warp load is one contiguous 512- or 256-byte run.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace cq {
+
+constexpr int TILE = 128;
+
+struct Dims {
+    int B, G;
+    int64_t N, K;
+    int NB, KT;       // tiles along N and K
+    int gpt;          // groups per tile = 128 / G
+    int code_bytes;   // bytes of the code part of a tile = 2048 * B
+    int tile_bytes;   // code_bytes + 128 * gpt * 8
+};
+
+__host__ __device__ inline Dims make_dims(int B, int G, int64_t N, int64_t K) {
+    Dims d;
+    d.B = B; d.G = G; d.N = N; d.K = K;
+    d.NB = (int)((N + TILE - 1) / TILE);
+    d.KT = (int)((K + TILE - 1) / TILE);
+    d.gpt = TILE / G;
+    d.code_bytes = 2048 * B;
+    d.tile_bytes = d.code_bytes + TILE * d.gpt * 8;
+    return d;
+}
+
+// ---- bit planes of the stored code u -------------------------------------------------------
+__host__ __device__ constexpr int plane_count(int B) { return (B == 3 || B == 5 || B == 6) ? 2 : (B == 7 ? 3 : 1); }
+__host__ __device__ constexpr int plane_width(int B, int i) {
+    return B == 1 ? 1 : B == 2 ? 2 : B == 3 ? (i == 0 ? 2 : 1) : B == 4 ? 4 : B == 5 ? (i == 0 ? 4 : 1)
+         : B == 6 ? (i == 0 ? 4 : 2) : B == 7 ? (i == 0 ? 4 : (i == 1 ? 2 : 1)) : 8;
+}
+__host__ __device__ constexpr int plane_bit_offset(int B, int i) {  // position of the plane inside u
+    return i == 0 ? 0 : (i == 1 ? plane_width(B, 0) : plane_width(B, 0) + plane_width(B, 1));
+}
+__host__ __device__ constexpr int plane_word_base(int B, int i) {   // first word of the plane in a lane record
+    return 2 * plane_bit_offset(B, i);
+}
+
+// byte offset of word W (0 .. 2B-1) of lane `lane` inside a row block
+__host__ __device__ inline int word_byte_offset(int B, int W, int lane) {
+    const int nfq = (2 * B) / 4;
+    if (W < 4 * nfq) return (((W >> 2) * 32) + lane) * 16 + (W & 3) * 4;
+    return nfq * 512 + lane * 8 + (W - 4 * nfq) * 4;
+}
+
+// Where weight (r, kk) of a tile lives: lane, pair index and half (0 = low 16 bits).
+struct Slot { int rb, lane, pair, half; };
+__host__ __device__ inline Slot slot_of(int r, int kk) {
+    Slot s;
+    const int rr = r & 15, g = rr & 7, hi_row = rr >> 3;
+    const int j = kk >> 4, kin = kk & 15, t = kin >> 2, sl = kin & 3;
+    s.rb = r >> 4;
+    s.lane = g * 4 + t;
+    s.pair = 4 * j + ((sl >> 1) * 2 + hi_row);
+    s.half = sl & 1;
+    return s;
+}
+// inverse: (rb, lane, pair, half) -> (r, kk)
+__host__ __device__ inline void weight_of(int rb, int lane, int pair, int half, int &r, int &kk) {
+    const int g = lane >> 2, t = lane & 3, j = pair >> 2, i = pair & 3;
+    r = rb * 16 + g + ((i & 1) ? 8 : 0);
+    kk = 16 * j + 4 * t + (i >> 1) * 2 + half;
+}
+
+struct __align__(8) GroupParams { float s; __half a; __half b; };
+
+__device__ __forceinline__ const uint8_t *tile_ptr(const void *layout, const Dims &d, int nb, int kb) {
+    return (const uint8_t *)layout + ((size_t)nb * d.KT + kb) * (size_t)d.tile_bytes;
+}
+
+// Slow generic accessor: stored code u of weight (n, k) (n < Np, k < Kp).
+__device__ inline unsigned fetch_u(const void *layout, const Dims &d, int64_t n, int64_t k) {
+    const int nb = (int)(n >> 7), kb = (int)(k >> 7);
+    const Slot s = slot_of((int)(n & 127), (int)(k & 127));
+    const uint8_t *rbp = tile_ptr(layout, d, nb, kb) + s.rb * 256 * d.B;
+    unsigned u = 0;
+    const int np = plane_count(d.B);
+    for (int i = 0; i < np; ++i) {
+        const int pw = plane_width(d.B, i), ppw = 16 / pw;
+        const int W = plane_word_base(d.B, i) + s.pair / ppw;
+        const int pos = (s.pair % ppw) * pw + 16 * s.half;
+        const uint32_t w = *(const uint32_t *)(rbp + word_byte_offset(d.B, W, s.lane));
+        u |= ((w >> pos) & ((1u << pw) - 1u)) << plane_bit_offset(d.B, i);
+    }
+    return u;
+}
+
+__device__ inline GroupParams fetch_params(const void *layout, const Dims &d, int64_t n, int64_t kgroup) {
+    const int nb = (int)(n >> 7), kb = (int)(kgroup / d.gpt), gi = (int)(kgroup % d.gpt);
+    const uint8_t *p = tile_ptr(layout, d, nb, kb) + d.code_bytes + (((int)(n & 127)) * d.gpt + gi) * 8;
+    return *(const GroupParams *)p;
+}
+
+// Signed code k from the stored code u (reserved pattern -> 0; W1: bit -> +-1).
+__host__ __device__ inline int signed_code(int B, unsigned u) {
+    if (B == 1) return u ? 1 : -1;
+    if (u == 0) return 0;
+    return (int)u - (1 << (B - 1));
+}
+
+// Normalised level q(i/M) by the Horner form of Eq. gpu-horner in fp32:
+//   t = i / M (IEEE division), c = (1 - a) - b, q = t * fma(t, fma(t, c, b), a).
+__device__ __forceinline__ float level_q(int i, int M, float a, float b) {
+    const float t = __fdiv_rn((float)i, (float)M);
+    const float c = __fsub_rn(__fsub_rn(1.0f, a), b);
+    return __fmul_rn(t, fmaf(t, fmaf(t, c, b), a));
+}
+
+// INT8 carrier of magnitude index i (Eq. carrier): RNE(127 q), clamped to [0, 127].
+// W1 / W2 have only the normalised levels {0, 1}, which sit on the carrier grid.
+__device__ __forceinline__ int carrier_of(int B, int i, float a, float b) {
+    if (B == 1) return 127;
+    if (B == 2) return i ? 127 : 0;
+    const int M = (1 << (B - 1)) - 1;
+    int r = __float2int_rn(__fmul_rn(127.0f, level_q(i, M, a, b)));
+    return min(max(r, 0), 127);
+}
+
+}  // namespace cq

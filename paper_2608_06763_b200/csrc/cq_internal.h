@@ -1,0 +1,41 @@
+// Internal launcher declarations shared by the translation units of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cq_common.cuh"
+
+namespace cq {
+
+cudaError_t launch_pack_codes(const int8_t *k, int B, int64_t N, int64_t K, uint8_t *codes, cudaStream_t st);
+cudaError_t launch_repack(const uint8_t *codes, const float *scale, const uint16_t *a, const uint16_t *b, const Dims &d,
+                          void *layout, cudaStream_t st);
+cudaError_t launch_unpack(const void *layout, const Dims &d, uint8_t *codes, float *scale, uint16_t *a, uint16_t *b,
+                          cudaStream_t st);
+cudaError_t launch_decode_levels(const void *layout, const Dims &d, float *levels, cudaStream_t st);
+cudaError_t launch_decode_carriers(const void *layout, const Dims &d, int8_t *carriers, cudaStream_t st);
+cudaError_t launch_decode_weights(const void *layout, const Dims &d, float *What, cudaStream_t st);
+cudaError_t launch_a8_partials(const void *layout, const Dims &d, const int8_t *x8, int64_t M, int32_t *P, cudaStream_t st);
+cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, int64_t x8_pitch, float *dx,
+                               cudaStream_t st);
+
+// Workspace carving (all offsets 256-byte aligned).
+struct Workspace {
+    size_t counters_off, counters_bytes;   // int32 arrival counters, one per 128-row block
+    size_t partial_off, partial_bytes;     // fp32 split-K partial sums [S][M][Np]
+    size_t x8_off, x8_bytes;               // Dynamic A8: int8 activation carrier [M][Kp]
+    size_t dx_off, dx_bytes;               // Dynamic A8: row scales [M]
+    size_t status_off;                     // int32 device status word (bounded waits report here)
+    size_t total;
+    int split_k;                           // S used by the small-M path
+};
+Workspace plan_workspace(const Dims &d, int64_t M, int mode);
+
+// Small-M (M <= 16) split-K tensor-core GEMV, both activation modes.
+cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
+                        uint8_t *ws, const Workspace &plan, cudaStream_t st);
+// Large-M tcgen05 / TMEM GEMM, both activation modes.
+cudaError_t launch_gemm_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
+                           uint8_t *ws, const Workspace &plan, cudaStream_t st);
+
+}  // namespace cq

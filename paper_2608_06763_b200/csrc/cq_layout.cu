@@ -1,0 +1,294 @@
+// Format kernels: canonical <-> device layout, debug decoders, and the Dynamic-A8 activation
+// quantiser.  All of them are one-time or test-side operations except cq::launch_quantize_a8.
+#include "cq_common.cuh"
+#include "cq_internal.h"
+
+namespace cq {
+
+// ---------------------------------------------------------------- canonical bitstream helpers
+// B-bit field j of a canonical row (Eq. gpu-packed-extraction): p = floor(jB/8), d = jB mod 8,
+// u = ((byte[p] >> d) | (byte[p+1] << (8-d))) & (2^B - 1).
+__device__ __forceinline__ unsigned canonical_field(const uint8_t *row, int64_t j, int B, int64_t row_bytes) {
+    const int64_t bit = j * B, p = bit >> 3;
+    const int dlt = (int)(bit & 7);
+    unsigned lo = row[p];
+    unsigned hi = (dlt + B > 8 && p + 1 < row_bytes) ? row[p + 1] : 0u;
+    return ((lo >> dlt) | (hi << (8 - dlt))) & ((1u << B) - 1u);
+}
+
+// canonical field -> stored code u (offset binary: the two's-complement sign bit flipped)
+__device__ __forceinline__ unsigned stored_from_field(int B, unsigned f) { return B == 1 ? f : (f ^ (1u << (B - 1))); }
+__device__ __forceinline__ unsigned field_from_stored(int B, unsigned u) { return B == 1 ? u : (u ^ (1u << (B - 1))); }
+
+// ---------------------------------------------------------------- cq_pack_codes
+// one thread per output byte: gathers the bits of the (up to 8) fields that touch it
+__global__ void pack_codes_kernel(const int8_t *__restrict__ k, int B, int64_t N, int64_t K, int64_t row_bytes,
+                                  uint8_t *__restrict__ codes) {
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= N * row_bytes) return;
+    const int64_t n = idx / row_bytes, byte = idx % row_bytes;
+    unsigned out = 0;
+    for (int bit = 0; bit < 8; ++bit) {
+        const int64_t bi = byte * 8 + bit, j = bi / B;
+        if (j >= K) break;
+        const int fb = (int)(bi % B);
+        const int code = k[n * K + j];
+        const unsigned field = (B == 1) ? (code > 0 ? 1u : 0u) : ((unsigned)code & ((1u << B) - 1u));
+        out |= ((field >> fb) & 1u) << bit;
+    }
+    codes[idx] = (uint8_t)out;
+}
+
+// ---------------------------------------------------------------- cq_repack
+// one thread per 32-bit code word of the layout
+__global__ void repack_codes_kernel(const uint8_t *__restrict__ codes, Dims d, int64_t row_bytes, uint8_t *__restrict__ layout) {
+    const int words_per_rb = 64 * d.B;   // 32 lanes * 2B words
+    const int words_per_tile = 8 * words_per_rb;
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t total = (int64_t)d.NB * d.KT * words_per_tile;
+    if (idx >= total) return;
+    const int64_t tile = idx / words_per_tile;
+    int rem = (int)(idx % words_per_tile);
+    const int rb = rem / words_per_rb; rem %= words_per_rb;
+    const int lane = rem / (2 * d.B), W = rem % (2 * d.B);
+    const int nb = (int)(tile / d.KT), kb = (int)(tile % d.KT);
+    // which plane does word W belong to
+    int pl = 0;
+    for (int i = plane_count(d.B) - 1; i > 0; --i) if (W >= plane_word_base(d.B, i)) { pl = i; break; }
+    const int pw = plane_width(d.B, pl), ppw = 16 / pw, bo = plane_bit_offset(d.B, pl);
+    const int wi = W - plane_word_base(d.B, pl);
+    uint32_t word = 0;
+    for (int q = 0; q < ppw; ++q) {
+        const int pair = wi * ppw + q;
+        for (int half = 0; half < 2; ++half) {
+            int r, kk;
+            weight_of(rb, lane, pair, half, r, kk);
+            const int64_t n = (int64_t)nb * TILE + r, k = (int64_t)kb * TILE + kk;
+            unsigned u;
+            if (n < d.N && k < d.K) u = stored_from_field(d.B, canonical_field(codes + n * row_bytes, k, d.B, row_bytes));
+            else u = (d.B == 1) ? 1u : (1u << (d.B - 1));  // padding: code 0 (W1: +1), its scale is 0
+            word |= ((u >> bo) & ((1u << pw) - 1u)) << (q * pw + 16 * half);
+        }
+    }
+    uint8_t *dst = layout + (size_t)tile * d.tile_bytes + rb * 256 * d.B + word_byte_offset(d.B, W, lane);
+    *(uint32_t *)dst = word;
+}
+
+// one thread per (tile, row, group-in-tile): parameter record, with the reserved-pattern flag
+__global__ void repack_params_kernel(const uint8_t *__restrict__ codes, const float *__restrict__ scale,
+                                     const uint16_t *__restrict__ a, const uint16_t *__restrict__ b, Dims d,
+                                     int64_t row_bytes, uint8_t *__restrict__ layout) {
+    const int per_tile = TILE * d.gpt;
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (int64_t)d.NB * d.KT * per_tile) return;
+    const int64_t tile = idx / per_tile;
+    const int rem = (int)(idx % per_tile), r = rem / d.gpt, gi = rem % d.gpt;
+    const int nb = (int)(tile / d.KT), kb = (int)(tile % d.KT);
+    const int64_t n = (int64_t)nb * TILE + r, kg = (int64_t)kb * d.gpt + gi, ng = d.K / d.G;
+    uint32_t sbits = 0;
+    uint16_t ha = 0x3C00, hb = 0;  // (1, 0)
+    if (n < d.N && kg < ng) {
+        sbits = __float_as_uint(scale[n * ng + kg]) & 0x7FFFFFFFu;
+        ha = a[n * ng + kg];
+        hb = b[n * ng + kg];
+        if (d.B > 1) {
+            bool reserved = false;
+            for (int j = 0; j < d.G; ++j)
+                reserved |= canonical_field(codes + n * row_bytes, kg * d.G + j, d.B, row_bytes) == (1u << (d.B - 1));
+            if (reserved) sbits |= 0x80000000u;
+        }
+    }
+    uint32_t *dst = (uint32_t *)(layout + (size_t)tile * d.tile_bytes + d.code_bytes + (r * d.gpt + gi) * 8);
+    dst[0] = sbits;
+    dst[1] = (uint32_t)ha | ((uint32_t)hb << 16);
+}
+
+// ---------------------------------------------------------------- cq_unpack
+// one thread per canonical byte
+__global__ void unpack_codes_kernel(const void *__restrict__ layout, Dims d, int64_t row_bytes, uint8_t *__restrict__ codes) {
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= d.N * row_bytes) return;
+    const int64_t n = idx / row_bytes, byte = idx % row_bytes;
+    unsigned out = 0;
+    int64_t last_j = -1;
+    unsigned field = 0;
+    for (int bit = 0; bit < 8; ++bit) {
+        const int64_t bi = byte * 8 + bit, j = bi / d.B;
+        if (j >= d.K) break;
+        if (j != last_j) { field = field_from_stored(d.B, fetch_u(layout, d, n, j)); last_j = j; }
+        out |= ((field >> (int)(bi % d.B)) & 1u) << bit;
+    }
+    codes[idx] = (uint8_t)out;
+}
+
+__global__ void unpack_params_kernel(const void *__restrict__ layout, Dims d, float *__restrict__ scale,
+                                     uint16_t *__restrict__ a, uint16_t *__restrict__ b) {
+    const int64_t ng = d.K / d.G;
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= d.N * ng) return;
+    const GroupParams p = fetch_params(layout, d, idx / ng, idx % ng);
+    scale[idx] = fabsf(p.s);
+    a[idx] = __half_as_ushort(p.a);
+    b[idx] = __half_as_ushort(p.b);
+}
+
+// ---------------------------------------------------------------- debug decoders
+// levels[N][K/G][L]: level_i = s * q(i/M) (Appendix B), fp32 Horner; W1: the scale
+__global__ void decode_levels_kernel(const void *__restrict__ layout, Dims d, float *__restrict__ levels) {
+    const int L = d.B == 1 ? 1 : (1 << (d.B - 1));
+    const int64_t ng = d.K / d.G;
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= d.N * ng * L) return;
+    const int i = (int)(idx % L);
+    const int64_t grp = idx / L;
+    const GroupParams p = fetch_params(layout, d, grp / ng, grp % ng);
+    const float s = fabsf(p.s);
+    float v;
+    if (d.B == 1) v = s;
+    else v = __fmul_rn(s, level_q(i, L - 1, __half2float(p.a), __half2float(p.b)));
+    levels[idx] = v;
+}
+
+__global__ void decode_carriers_kernel(const void *__restrict__ layout, Dims d, int8_t *__restrict__ carriers) {
+    const int L = d.B == 1 ? 1 : (1 << (d.B - 1));
+    const int64_t ng = d.K / d.G;
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= d.N * ng * L) return;
+    const int i = (int)(idx % L);
+    const int64_t grp = idx / L;
+    const GroupParams p = fetch_params(layout, d, grp / ng, grp % ng);
+    carriers[idx] = (int8_t)carrier_of(d.B, i, __half2float(p.a), __half2float(p.b));
+}
+
+__global__ void decode_weights_kernel(const void *__restrict__ layout, Dims d, float *__restrict__ What) {
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= d.N * d.K) return;
+    const int64_t n = idx / d.K, k = idx % d.K;
+    const int code = signed_code(d.B, fetch_u(layout, d, n, k));
+    const GroupParams p = fetch_params(layout, d, n, k / d.G);
+    const float s = fabsf(p.s);
+    float v;
+    if (d.B == 1) v = s;
+    else {
+        const int M = (1 << (d.B - 1)) - 1;
+        v = __fmul_rn(s, level_q(abs(code), M, __half2float(p.a), __half2float(p.b)));
+    }
+    What[idx] = code < 0 ? -v : (code == 0 ? 0.0f : v);
+}
+
+// P[M][N][K/G] = sum_{j in g} x8[m][j] * r(k_j)   (Eq. a8-output), one thread per partial
+__global__ void a8_partials_kernel(const void *__restrict__ layout, Dims d, const int8_t *__restrict__ x8, int64_t M,
+                                   int32_t *__restrict__ P) {
+    const int64_t ng = d.K / d.G;
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= M * d.N * ng) return;
+    const int64_t g = idx % ng, n = (idx / ng) % d.N, m = idx / (ng * d.N);
+    const GroupParams p = fetch_params(layout, d, n, g);
+    const float a = __half2float(p.a), b = __half2float(p.b);
+    int acc = 0;
+    for (int j = 0; j < d.G; ++j) {
+        const int64_t k = g * d.G + j;
+        const int code = signed_code(d.B, fetch_u(layout, d, n, k));
+        int r = code == 0 ? 0 : carrier_of(d.B, abs(code), a, b);
+        if (code < 0) r = -r;
+        acc += (int)x8[m * d.K + k] * r;
+    }
+    P[idx] = acc;
+}
+
+// ---------------------------------------------------------------- Dynamic-A8 activation quantiser
+// One block per row (Eq. a8-activation-scale, Eq. a8-activation-quantization).  fp32 arithmetic:
+// xbar = max(max|x|, 1e-10f); dx = xbar / 127 (IEEE); x8 = clip(round-half-away(x / dx), +-127).
+// Written with a row pitch so the GEMM can ask for a padded carrier.
+__global__ void __launch_bounds__(256) quantize_a8_kernel(const uint16_t *__restrict__ x, int64_t M, int64_t K,
+                                                         int8_t *__restrict__ x8, int64_t x8_pitch,
+                                                         float *__restrict__ dx) {
+    __shared__ float red[8];
+    __shared__ float s_d;
+    const int64_t m = blockIdx.x;
+    const uint16_t *row = x + m * K;
+    float mx = 0.0f;
+    for (int64_t j = threadIdx.x; j < K; j += blockDim.x)
+        mx = fmaxf(mx, fabsf(__uint_as_float((uint32_t)row[j] << 16)));
+    for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float v = red[0];
+        for (int i = 1; i < (int)(blockDim.x >> 5); ++i) v = fmaxf(v, red[i]);
+        v = fmaxf(v, 1e-10f);
+        const float d = __fdiv_rn(v, 127.0f);
+        s_d = d;
+        dx[m] = d;
+    }
+    __syncthreads();
+    const float d = s_d;
+    int8_t *orow = x8 + m * x8_pitch;
+    for (int64_t j = threadIdx.x; j < x8_pitch; j += blockDim.x) {
+        int q = 0;
+        if (j < K) {
+            const float v = __fdiv_rn(__uint_as_float((uint32_t)row[j] << 16), d);
+            float r = roundf(v);  // halves away from zero
+            r = fminf(fmaxf(r, -127.0f), 127.0f);
+            q = (int)r;
+        }
+        orow[j] = (int8_t)q;
+    }
+}
+
+// ---------------------------------------------------------------- launchers
+static inline unsigned blocks_for(int64_t n, int t) { return (unsigned)((n + t - 1) / t); }
+
+cudaError_t launch_pack_codes(const int8_t *k, int B, int64_t N, int64_t K, uint8_t *codes, cudaStream_t st) {
+    const int64_t rbts = (K * B + 7) / 8;
+    pack_codes_kernel<<<blocks_for(N * rbts, 256), 256, 0, st>>>(k, B, N, K, rbts, codes);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_repack(const uint8_t *codes, const float *scale, const uint16_t *a, const uint16_t *b, const Dims &d,
+                          void *layout, cudaStream_t st) {
+    const int64_t rbts = (d.K * d.B + 7) / 8;
+    const int64_t words = (int64_t)d.NB * d.KT * 8 * 64 * d.B;
+    repack_codes_kernel<<<blocks_for(words, 256), 256, 0, st>>>(codes, d, rbts, (uint8_t *)layout);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int64_t recs = (int64_t)d.NB * d.KT * TILE * d.gpt;
+    repack_params_kernel<<<blocks_for(recs, 256), 256, 0, st>>>(codes, scale, a, b, d, rbts, (uint8_t *)layout);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_unpack(const void *layout, const Dims &d, uint8_t *codes, float *scale, uint16_t *a, uint16_t *b,
+                          cudaStream_t st) {
+    const int64_t rbts = (d.K * d.B + 7) / 8;
+    unpack_codes_kernel<<<blocks_for(d.N * rbts, 256), 256, 0, st>>>(layout, d, rbts, codes);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    unpack_params_kernel<<<blocks_for(d.N * (d.K / d.G), 256), 256, 0, st>>>(layout, d, scale, a, b);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decode_levels(const void *layout, const Dims &d, float *levels, cudaStream_t st) {
+    const int L = d.B == 1 ? 1 : (1 << (d.B - 1));
+    decode_levels_kernel<<<blocks_for(d.N * (d.K / d.G) * L, 256), 256, 0, st>>>(layout, d, levels);
+    return cudaGetLastError();
+}
+cudaError_t launch_decode_carriers(const void *layout, const Dims &d, int8_t *carriers, cudaStream_t st) {
+    const int L = d.B == 1 ? 1 : (1 << (d.B - 1));
+    decode_carriers_kernel<<<blocks_for(d.N * (d.K / d.G) * L, 256), 256, 0, st>>>(layout, d, carriers);
+    return cudaGetLastError();
+}
+cudaError_t launch_decode_weights(const void *layout, const Dims &d, float *What, cudaStream_t st) {
+    decode_weights_kernel<<<blocks_for(d.N * d.K, 256), 256, 0, st>>>(layout, d, What);
+    return cudaGetLastError();
+}
+cudaError_t launch_a8_partials(const void *layout, const Dims &d, const int8_t *x8, int64_t M, int32_t *P, cudaStream_t st) {
+    a8_partials_kernel<<<blocks_for(M * d.N * (d.K / d.G), 128), 128, 0, st>>>(layout, d, x8, M, P);
+    return cudaGetLastError();
+}
+cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, int64_t x8_pitch, float *dx,
+                               cudaStream_t st) {
+    quantize_a8_kernel<<<(unsigned)M, 256, 0, st>>>(x, M, K, x8, x8_pitch, dx);
+    return cudaGetLastError();
+}
+
+}  // namespace cq

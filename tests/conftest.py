@@ -12,6 +12,11 @@ GOLDEN = os.path.join(ROOT, "tests", "golden")
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (sm_100a)")
+    # build the CUDA library (nvcc cross-compiles without a GPU) and the C oracle if they are stale
+    from paper_2608_06763_b200.build import build
+    build()
+    import oracle
+    oracle.build()
 
 
 def read_table(name):

@@ -1,0 +1,57 @@
+"""The C-ABI library loads and exports every symbol include/cubicquant.h declares; host-side
+size functions and argument validation (no compute, no GPU)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2608_06763_b200 as cq
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "cubicquant.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(cq_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    L = cq.lib()
+    names = declared_functions()
+    assert len(names) >= 16
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_sizes():
+    assert cq.cq_canonical_code_bytes(4, 4096, 4096) == 4096 * 2048
+    assert cq.cq_canonical_code_bytes(3, 2, 40) == 2 * 15
+    # device layout has exactly the canonical byte count when N and K are multiples of 128
+    for B in range(1, 9):
+        for G in (32, 64, 128):
+            assert cq.cq_layout_bytes(B, G, 256, 384) == 256 * 384 * B // 8 + 256 * (384 // G) * 8
+            assert cq.cq_effective_bits(B, G) == B + 64 / G
+    assert cq.cq_layout_bytes(4, 128, 130, 128) == 2 * (128 * 128 // 2 + 128 * 8)  # N padded to 256
+    assert cq.cq_layout_bytes(4, 48, 128, 96) == 0 and cq.cq_layout_bytes(4, 128, 128, 192) == 0
+    assert cq.cq_workspace_bytes(4, 128, 1, 4096, 4096, cq.CQ_MODEL_DTYPE) > 0
+    assert cq.cq_workspace_bytes(4, 128, 1, 4096, 4096, cq.CQ_DYN_A8) > cq.cq_workspace_bytes(4, 128, 1, 4096, 4096, 0)
+    assert cq.cq_workspace_bytes(4, 128, 1, 4096, 4096, 7) == 0
+
+
+def test_argument_errors_are_found_before_any_launch():
+    L = cq.lib()
+    one = ctypes.c_void_p(16)  # non-null, aligned, never dereferenced: validation fails first
+    odd = ctypes.c_void_p(24)
+    assert L.cq_gemm(None, 4, 128, one, one, 1, 128, 128, 0, one, 1 << 20, None) == -1
+    assert L.cq_gemm(one, 9, 128, one, one, 1, 128, 128, 0, one, 1 << 20, None) == -1
+    assert L.cq_gemm(one, 4, 128, one, one, 0, 128, 128, 0, one, 1 << 20, None) == -1
+    assert L.cq_gemm(one, 4, 128, one, one, 1, 128, 128, 5, one, 1 << 20, None) == -1
+    assert L.cq_gemm(one, 4, 128, one, one, 1, 128, 192, 0, one, 1 << 20, None) == -2   # K % G != 0
+    assert L.cq_gemm(one, 4, 256, one, one, 1, 128, 256, 0, one, 1 << 20, None) == -2   # G unsupported
+    assert L.cq_gemm(one, 4, 128, odd, one, 1, 128, 128, 0, one, 1 << 20, None) == -3
+    assert L.cq_gemm(one, 4, 128, one, one, 1, 128, 128, 0, one, 16, None) == -4        # workspace too small
+    assert L.cq_repack(None, one, one, one, 4, 128, 128, 128, one, None) == -1
+    assert L.cq_quantize_a8(one, 0, 128, one, one, None) == -1
+    assert cq.cq_status_string(-4) == "CQ_ERR_WORKSPACE"

@@ -1,0 +1,97 @@
+"""GPU parity of cq_gemm against the oracle at sizes the oracle finishes in seconds: every width,
+every group size, both modes, M across the small-M / large-M boundary, ragged N and K."""
+import numpy as np
+import pytest
+import torch
+
+import datagen
+import oracle
+import paper_2608_06763_b200 as cq
+from util import Case, check_y, encoded_case, logical_case, x_to_device, y_to_numpy
+
+pytestmark = pytest.mark.gpu
+
+ALL_B = [1, 2, 3, 4, 5, 6, 7, 8]
+
+
+def run_both(c, x_bits, mode):
+    y = y_to_numpy(cq.cq_gemm(c.pw, x_to_device(x_bits), mode))
+    if mode == cq.CQ_MODEL_DTYPE:
+        ref = oracle.gemm_model(c.codes, c.s, c.a, c.b, c.B, c.G, c.K, x_bits)
+    else:
+        x8, dx = oracle.quantize_a8(x_bits)
+        ref = oracle.gemm_a8(c.codes, c.s, c.a, c.b, c.B, c.G, c.K, x8, dx)
+    return y, ref
+
+
+@pytest.mark.parametrize("mode", [cq.CQ_MODEL_DTYPE, cq.CQ_DYN_A8])
+@pytest.mark.parametrize("G", [32, 64, 128])
+@pytest.mark.parametrize("B", ALL_B)
+def test_gemv_m1_all_widths_and_groups(B, G, mode):
+    c = encoded_case("laplace", 384, 1024, B, G, seed=100 + B, b=0.015)
+    x = datagen.activations(1, 1024, seed=101)
+    y, ref = run_both(c, x, mode)
+    check_y(y, ref, f"B={B} G={G} mode={mode}")
+
+
+@pytest.mark.parametrize("mode", [cq.CQ_MODEL_DTYPE, cq.CQ_DYN_A8])
+@pytest.mark.parametrize("M", [1, 3, 8, 9, 16])
+def test_small_m_rows(M, mode):
+    c = encoded_case("outlier", 256, 2048, 4, 128, seed=110, sigma=0.02, sigma_out=0.2, p=0.001)
+    x = datagen.activations(M, 2048, seed=111, outlier_cols=0.01)
+    y, ref = run_both(c, x, mode)
+    check_y(y, ref, f"M={M} mode={mode}")
+
+
+@pytest.mark.parametrize("mode", [cq.CQ_MODEL_DTYPE, cq.CQ_DYN_A8])
+@pytest.mark.parametrize("B", [2, 3, 4, 8])
+def test_ragged_shapes_and_reserved_codes(B, mode):
+    # N and K not multiples of the 128 tile, K not a multiple of 8 elements per row is not allowed by
+    # K % G == 0, so the ragged K case is K = 3 * 32 + 128 ... = 224 (G = 32)
+    N, K, G = 200, 224, 32
+    c = logical_case(N, K, B, G, seed=120 + B)
+    c.k[7, 10:20] = -(1 << (B - 1))  # reserved pattern decodes to zero
+    c.k[150, :] = 0
+    c.s[9, 2] = 0.0                   # all-zero group
+    c = Case(c.k, c.s, c.a, c.b, B, G)
+    x = datagen.activations(5, K, seed=121)
+    y, ref = run_both(c, x, mode)
+    check_y(y, ref, f"ragged B={B} mode={mode}")
+    assert np.all(y[:, 150] == 0.0)
+
+
+@pytest.mark.parametrize("mode", [cq.CQ_MODEL_DTYPE, cq.CQ_DYN_A8])
+def test_extreme_activation_magnitudes(mode):
+    # rows with huge and tiny magnitudes: the per-row scaling must neither overflow nor flush
+    c = encoded_case("normal", 128, 512, 4, 128, seed=130)
+    x = datagen.bf16_bits_to_f32(datagen.activations(4, 512, seed=131)).copy()
+    x[0] *= 3.0e4
+    x[1] *= 1.0e-6
+    x[2, :] = 0.0
+    x[3, 17] = 5.0e5
+    xb = datagen.to_bf16_bits(x)
+    y, ref = run_both(c, xb, mode)
+    for m in range(4):
+        if m == 2:
+            assert np.all(y[m] == 0)
+        else:
+            check_y(y[m:m + 1], ref[m:m + 1], f"row {m} mode={mode}")
+
+
+@pytest.mark.parametrize("mode", [cq.CQ_MODEL_DTYPE, cq.CQ_DYN_A8])
+@pytest.mark.parametrize("M", [17, 64, 129, 300])
+@pytest.mark.parametrize("B", [3, 4, 8])
+def test_large_m_rows(B, M, mode):
+    c = encoded_case("normal", 256, 1024, B, 128, seed=140 + B, sigma=0.015)
+    x = datagen.activations(M, 1024, seed=141, outlier_cols=0.01)
+    y, ref = run_both(c, x, mode)
+    check_y(y, ref, f"B={B} M={M} mode={mode}")
+
+
+def test_repeatable_bitwise_and_workspace_reuse():
+    c = encoded_case("normal", 512, 4096, 4, 128, seed=150)
+    x = x_to_device(datagen.activations(4, 4096, seed=151))
+    ws = torch.zeros(cq.cq_workspace_bytes(4, 128, 4, 512, 4096, 0), dtype=torch.uint8, device="cuda")
+    y1 = cq.cq_gemm(c.pw, x, 0, ws).clone()
+    y2 = cq.cq_gemm(c.pw, x, 0, ws).clone()
+    assert torch.equal(y1.view(torch.int16), y2.view(torch.int16))  # fixed split-K order: deterministic
