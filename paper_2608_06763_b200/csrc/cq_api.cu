@@ -10,20 +10,19 @@ namespace cq {
 
 static thread_local int g_last_cuda_error = 0;
 
-int gemv_split_k(const Dims &d);
 int gemm_tc_available();
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 Workspace plan_workspace(const Dims &d, int64_t M, int mode) {
     Workspace w{};
-    const int64_t Np = (int64_t)d.NB * TILE, Kp = (int64_t)d.KT * TILE;
+    const int64_t Kp = (int64_t)d.KT * TILE;
     const int64_t Mc = M < 16 ? M : 16;  // rows handled by one small-M launch
-    w.split_k = gemv_split_k(d);
+    const GemvPlan gp = gemv_plan(d, Mc);
     size_t off = 0;
     w.counters_off = off; w.counters_bytes = align_up((size_t)d.NB * 4, 256); off += w.counters_bytes;
     w.status_off = off; off += 256;
-    w.partial_off = off; w.partial_bytes = align_up((size_t)w.split_k * Mc * Np * 4, 256); off += w.partial_bytes;
+    w.partial_off = off; w.partial_bytes = align_up((size_t)d.NB * gp.max_slots * Mc * TILE * 4, 256); off += w.partial_bytes;
     if (mode == CQ_DYN_A8) {
         w.x8_off = off; w.x8_bytes = align_up((size_t)(M + 127) / 128 * 128 * Kp, 256); off += w.x8_bytes;
         w.dx_off = off; w.dx_bytes = align_up((size_t)M * 4, 256); off += w.dx_bytes;

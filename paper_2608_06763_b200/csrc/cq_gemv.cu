@@ -1,16 +1,24 @@
-// Small-M (M <= 16) packed GEMV: split-K, weights streamed exactly once, warp-level tensor-core
-// MMAs doing the multiply and the k reduction (Section 5.3 narrow-row path; Section 5.4 for A8).
+// Small-M (M <= 16) packed GEMV: weights streamed exactly once, warp-level tensor-core MMAs doing
+// the multiply and the k reduction (Section 5.3 narrow-row path; Section 5.4 for Dynamic A8).
 //
-// Work decomposition: CTA = one 128-row block x one K slice; its 8 warps own the 8 row blocks of
-// 16 rows.  A lane's 128-bit loads land directly in its MMA A-fragment positions (see
-// cq_common.cuh), so decode is: mask two codes out of a word, turn them into fp16 by the
-// exponent-bias trick, evaluate the group's cubic in half2 Horner form (Eq. gpu-horner) on the
-// power-of-two-normalised code, and feed the MMA.  The group scale s_g is applied to the fp32
-// group reduction, as the paper's narrow path does.  Activations are converted bf16 -> fp16 with
-// a per-token power-of-two scale chosen per CTA so that nothing overflows or loses bits.
+// Work decomposition (balanced, persistent): the NB x KT grid of 128 x 128 weight tiles is cut
+// into P equal contiguous runs (P = resident CTAs of the whole GPU), one per CTA, in row-block
+// major order.  A run covers one or more row blocks; for each it streams its K range, and either
+// writes y (it covered the whole K range) or a partial sum into its slot; the last CTA to arrive
+// at a row block adds the slots in slot order (deterministic) and writes y.  The 8 warps of a CTA
+// own the 8 groups of 16 rows of a tile.
+//
+// Decode: a lane's 128-bit loads land directly in its MMA A-fragment positions (cq_common.cuh).
+// Two codes are masked out of a word straight into fp16 mantissas (exponent-bias trick), one exact
+// FMA turns them into the normalised signed code T = k / 2^(B-1), and the group's cubic is
+// evaluated in half2 Horner form (Eq. gpu-horner) as T (a' + |T| (b' + |T| c')).  The group scale
+// s_g multiplies the fp32 group reduction, as in the paper's narrow path.  Activations go
+// bf16 -> fp16 with a per-token power-of-two scale so that nothing overflows or loses bits.
 //
 // Dynamic A8 uses the INT8 m16n8k32 MMA on signed carriers looked up in a per-warp table of the
 // group's non-negative carriers (Eq. carrier), int32 group partials, fp32 rescale (Eq. a8-output).
+#include <utility>
+
 #include "cq_common.cuh"
 #include "cq_internal.h"
 
@@ -19,8 +27,17 @@ namespace cq {
 namespace {
 
 constexpr int GEMV_THREADS = 256;
-constexpr int XS_PAD = 16;          // halves of padding per staged activation row (bank spread)
-constexpr int MAX_SLICE_TILES = 16; // K tiles per CTA at most (bounds shared memory)
+constexpr int XS_PAD = 16;     // elements of padding per staged activation row (bank spread)
+constexpr int MAX_SUB = 16;    // K tiles staged at a time (bounds shared memory)
+
+template <int... I, class F>
+__device__ __forceinline__ void static_for_impl(F &&f, std::integer_sequence<int, I...>) {
+    (f(std::integral_constant<int, I>{}), ...);
+}
+template <int N, class F>
+__device__ __forceinline__ void static_for(F &&f) {
+    static_for_impl(static_cast<F &&>(f), std::make_integer_sequence<int, N>{});
+}
 
 __device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -46,11 +63,23 @@ __device__ __forceinline__ uint2 ld_stream8(const void *p) {
     return v;
 }
 
-template <int B>
-struct Rec { uint32_t w[2 * B]; };
+// fp16 bit patterns built with integer arithmetic only (so they are compile-time constants)
+constexpr uint32_t h2dup(uint32_t h) { return h | (h << 16); }
+constexpr uint32_t half_pow2(int e) { return (uint32_t)((e + 15) << 10); }                      // 2^e, -14 <= e <= 15
+constexpr uint32_t half_neg_pow2_plus(int q, int c) {                                            // -(2^q + c), c < 2^q, q <= 10
+    return 0x8000u | (uint32_t)((q + 15) << 10) | (uint32_t)(c << (10 - q));
+}
+__device__ __forceinline__ __half2 as_h2(uint32_t v) { return *reinterpret_cast<__half2 *>(&v); }
+__device__ __forceinline__ uint32_t as_u32(__half2 v) { return *reinterpret_cast<uint32_t *>(&v); }
 
-template <int B>
-__device__ __forceinline__ void load_rec(Rec<B> &r, const uint8_t *rbp, int lane) {
+template <int B, int GPT>
+struct TileRegs {
+    uint32_t w[2 * B];
+    uint2 prm[2][GPT];  // {s bits, a | b << 16} of rows g and g + 8
+};
+
+template <int B, int GPT>
+__device__ __forceinline__ void load_tile(TileRegs<B, GPT> &r, const uint8_t *rbp, const uint8_t *prm, int lane) {
     constexpr int NFQ = (2 * B) / 4;
 #pragma unroll
     for (int q = 0; q < NFQ; ++q) {
@@ -61,48 +90,51 @@ __device__ __forceinline__ void load_rec(Rec<B> &r, const uint8_t *rbp, int lane
         const uint2 v = ld_stream8(rbp + NFQ * 512 + lane * 8);
         r.w[4 * NFQ + 0] = v.x; r.w[4 * NFQ + 1] = v.y;
     }
+#pragma unroll
+    for (int gi = 0; gi < GPT; ++gi) {
+        r.prm[0][gi] = ld_stream8(prm + gi * 8);
+        r.prm[1][gi] = ld_stream8(prm + (8 * GPT + gi) * 8);
+    }
 }
 
-// Two stored codes of pair p as packed 16-bit integers (u_lo | u_hi << 16).  Generic form.
-template <int B>
-__device__ __forceinline__ uint32_t pair_codes(const uint32_t (&w)[2 * B], int p) {
+// Two stored codes of pair P as packed 16-bit integers (u_lo | u_hi << 16).
+template <int B, int P>
+__device__ __forceinline__ uint32_t pair_codes(const uint32_t (&w)[2 * B]) {
     uint32_t u2 = 0;
-#pragma unroll
-    for (int i = 0; i < plane_count(B); ++i) {
-        const int pw = plane_width(B, i), ppw = 16 / pw;
-        const int W = plane_word_base(B, i) + p / ppw, pos = (p % ppw) * pw;
-        const uint32_t m = ((1u << pw) - 1u) * 0x00010001u;
+    static_for<plane_count(B)>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        constexpr int pw = plane_width(B, i), ppw = 16 / pw;
+        constexpr int W = plane_word_base(B, i) + P / ppw, pos = (P % ppw) * pw;
+        constexpr uint32_t m = ((1u << pw) - 1u) * 0x00010001u;
         u2 |= ((w[W] >> pos) & m) << plane_bit_offset(B, i);
-    }
+    });
     return u2;
 }
 
-// Pair p as half2 of the normalised signed code:  B >= 3: k / 2^(B-1);  B = 2: k;  B = 1: k (+-1).
-// The stored code lands in the fp16 mantissa under exponent bits 0x6400 (value 1024 + u * 2^pos);
+// Pair P as half2 of the normalised signed code:  B >= 3: T = k / 2^(B-1);  B <= 2: k itself.
+// The stored code lands in the fp16 mantissa under exponent bits 0x6400 (value 1024 + u 2^pos);
 // one exact FMA removes the offset and the position scale.
-template <int B>
-__device__ __forceinline__ __half2 pair_T(const uint32_t (&w)[2 * B], int p) {
+template <int B, int P>
+__device__ __forceinline__ __half2 pair_T(const uint32_t (&w)[2 * B]) {
     if constexpr (plane_count(B) == 1) {
-        constexpr int PPW = 16 / B;
-        const int W = p / PPW;
-        int pos = (p % PPW) * B;
-        uint32_t word = w[W];
-        if constexpr (B == 1) {  // keep the field off mantissa bit 0 so the offset constant stays representable
-            if (pos <= 6) { word <<= 1; pos += 1; } else { word >>= 6; pos -= 6; }
-        } else {
-            if (pos + B > 10) { word >>= 8; pos -= 8; }
-        }
-        const uint32_t m = (((1u << B) - 1u) << pos) * 0x00010001u;
+        constexpr int PPW = 16 / B, W = P / PPW, pos0 = (P % PPW) * B;
+        // B = 1 keeps the field off mantissa bit 0 (the offset constant must stay representable);
+        // other widths shift by 8 when the field would leave the 10 mantissa bits
+        constexpr int shl = (B == 1 && pos0 <= 6) ? 1 : 0;
+        constexpr int shr = (B == 1) ? (pos0 <= 6 ? 0 : 6) : (pos0 + B > 10 ? 8 : 0);
+        constexpr int pos = pos0 + shl - shr;
+        const uint32_t word = shl ? (w[W] << shl) : (shr ? (w[W] >> shr) : w[W]);
+        constexpr uint32_t m = (((1u << B) - 1u) << pos) * 0x00010001u;
         const uint32_t hbits = (word & m) | 0x64006400u;
-        float sc, off;
-        if constexpr (B == 1) { sc = exp2f((float)(1 - pos)); off = -(exp2f((float)(11 - pos)) + 1.0f); }
-        else if constexpr (B == 2) { sc = exp2f((float)(-pos)); off = -(exp2f((float)(10 - pos)) + 2.0f); }
-        else { sc = exp2f((float)(-(pos + B - 1))); off = -(exp2f((float)(10 - pos - (B - 1))) + 1.0f); }
-        return __hfma2(*reinterpret_cast<const __half2 *>(&hbits), __float2half2_rn(sc), __float2half2_rn(off));
+        constexpr uint32_t sc = (B == 1) ? half_pow2(1 - pos) : (B == 2) ? half_pow2(-pos) : half_pow2(-(pos + B - 1));
+        constexpr uint32_t off = (B == 1) ? half_neg_pow2_plus(11 - pos, 1)
+                               : (B == 2) ? half_neg_pow2_plus(10 - pos, 2)
+                                          : half_neg_pow2_plus(10 - pos - (B - 1), 1);
+        return __hfma2(as_h2(hbits), as_h2(h2dup(sc)), as_h2(h2dup(off)));
     } else {
-        const uint32_t hbits = pair_codes<B>(w, p) | 0x64006400u;
-        const float sc = exp2f((float)(-(B - 1))), off = -(exp2f((float)(10 - (B - 1))) + 1.0f);
-        return __hfma2(*reinterpret_cast<const __half2 *>(&hbits), __float2half2_rn(sc), __float2half2_rn(off));
+        const uint32_t hbits = pair_codes<B, P>(w) | 0x64006400u;
+        constexpr uint32_t sc = half_pow2(-(B - 1)), off = half_neg_pow2_plus(10 - (B - 1), 1);
+        return __hfma2(as_h2(hbits), as_h2(h2dup(sc)), as_h2(h2dup(off)));
     }
 }
 
@@ -111,15 +143,17 @@ struct RowCoef { __half2 a2, b2, c2; float s; };
 // Coefficients of q as a polynomial in T = k / 2^(B-1):  t = |T| rho, rho = 2^(B-1) / M, so
 // q = |T| (a rho + |T| (b rho^2 + |T| c rho^3)).
 template <int B>
-__device__ __forceinline__ RowCoef make_coef(const GroupParams &p) {
+__device__ __forceinline__ RowCoef make_coef(uint2 p) {
     RowCoef c;
-    c.s = fabsf(p.s);
+    c.s = __uint_as_float(p.x & 0x7FFFFFFFu);
     if constexpr (B >= 3) {
         constexpr float rho = (float)(1 << (B - 1)) / (float)((1 << (B - 1)) - 1);
-        const float a = __half2float(p.a), b = __half2float(p.b), cc = (1.0f - a) - b;
+        constexpr float rho2 = rho * rho, rho3 = rho * rho * rho;
+        const __half2 ab = as_h2(p.y);
+        const float a = __low2float(ab), b = __high2float(ab), cc = (1.0f - a) - b;
         c.a2 = __float2half2_rn(a * rho);
-        c.b2 = __float2half2_rn(b * rho * rho);
-        c.c2 = __float2half2_rn(cc * rho * rho * rho);
+        c.b2 = __float2half2_rn(b * rho2);
+        c.c2 = __float2half2_rn(cc * rho3);
     }
     return c;
 }
@@ -130,343 +164,372 @@ __device__ __forceinline__ uint32_t level_pair(__half2 T, const RowCoef &c) {
         const __half2 bad = __float2half2_rn(B == 2 ? -2.0f : -1.0f);
         T = __hmul2(T, __hne2(T, bad));
     }
-    __half2 v;
     if constexpr (B >= 3) {
         const __half2 at = __habs2(T);
-        v = __hmul2(T, __hfma2(at, __hfma2(at, c.c2, c.b2), c.a2));
+        return as_u32(__hmul2(T, __hfma2(at, __hfma2(at, c.c2, c.b2), c.a2)));
     } else {
-        v = T;
+        return as_u32(T);
     }
-    return *reinterpret_cast<uint32_t *>(&v);
 }
+
+// One group of a tile, model dtype: CPG MMAs per token block into D, then acc += s * D.
+template <int B, int G, int NT, int GI, bool FIX>
+__device__ __forceinline__ void group_model(const TileRegs<B, TILE / G> &r, const __half *xl, int XS, float (&acc)[NT][4]) {
+    constexpr int CPG = G / 16;
+    const RowCoef c_lo = make_coef<B>(r.prm[0][GI]), c_hi = make_coef<B>(r.prm[1][GI]);
+    float D[NT][4];
+#pragma unroll
+    for (int tb = 0; tb < NT; ++tb)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) D[tb][i] = 0.0f;
+    static_for<CPG>([&](auto jc) {
+        constexpr int j = GI * CPG + decltype(jc)::value;
+        uint32_t A[4];
+        A[0] = level_pair<B, FIX>(pair_T<B, 4 * j + 0>(r.w), c_lo);
+        A[1] = level_pair<B, FIX>(pair_T<B, 4 * j + 1>(r.w), c_hi);
+        A[2] = level_pair<B, FIX>(pair_T<B, 4 * j + 2>(r.w), c_lo);
+        A[3] = level_pair<B, FIX>(pair_T<B, 4 * j + 3>(r.w), c_hi);
+#pragma unroll
+        for (int tb = 0; tb < NT; ++tb) {
+            const uint2 bf = *(const uint2 *)(xl + tb * 8 * XS + 16 * j);
+            mma_f16(D[tb], A, bf.x, bf.y);
+        }
+    });
+#pragma unroll
+    for (int tb = 0; tb < NT; ++tb) {
+        acc[tb][0] = fmaf(c_lo.s, D[tb][0], acc[tb][0]);
+        acc[tb][1] = fmaf(c_lo.s, D[tb][1], acc[tb][1]);
+        acc[tb][2] = fmaf(c_hi.s, D[tb][2], acc[tb][2]);
+        acc[tb][3] = fmaf(c_hi.s, D[tb][3], acc[tb][3]);
+    }
+}
+
+// One group of a tile, Dynamic A8: carriers from the warp's table, INT8 MMAs, acc += s * P_g.
+template <int B, int G, int NT, int GI>
+__device__ __forceinline__ void group_a8(const TileRegs<B, TILE / G> &r, const int8_t *xl, int XS, int8_t *ctab, int g,
+                                         int t, float (&acc)[NT][4]) {
+    constexpr int CPG = G / 16;
+    constexpr int L = B == 1 ? 1 : (1 << (B - 1));
+    const uint2 p_lo = r.prm[0][GI], p_hi = r.prm[1][GI];
+    if constexpr (B >= 3) {  // lane (g, t) fills entries i = t mod 4 of rows g and g + 8
+        __syncwarp();
+        const __half2 ab_lo = as_h2(p_lo.y), ab_hi = as_h2(p_hi.y);
+        const float a_lo = __low2float(ab_lo), b_lo = __high2float(ab_lo);
+        const float a_hi = __low2float(ab_hi), b_hi = __high2float(ab_hi);
+        for (int i = t; i < L; i += 4) {
+            ctab[g * L + i] = (int8_t)carrier_of(B, i, a_lo, b_lo);
+            ctab[(g + 8) * L + i] = (int8_t)carrier_of(B, i, a_hi, b_hi);
+        }
+        __syncwarp();
+    }
+    int D[NT][4];
+#pragma unroll
+    for (int tb = 0; tb < NT; ++tb)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) D[tb][i] = 0;
+    static_for<CPG / 2>([&](auto jc) {
+        constexpr int j = GI * CPG + 2 * decltype(jc)::value;
+        uint32_t A[4];
+        // a0: row g chunk j; a1: row g+8 chunk j; a2: row g chunk j+1; a3: row g+8 chunk j+1
+        static_for<4>([&](auto rc) {
+            constexpr int rr = decltype(rc)::value, jcx = j + (rr >> 1), hi_row = rr & 1;
+            uint32_t packed = 0;
+            static_for<2>([&](auto ec) {  // pairs (hi_row) and (2 + hi_row) hold k+0,1 and k+2,3
+                constexpr int e = decltype(ec)::value;
+                const uint32_t u2 = pair_codes<B, 4 * jcx + 2 * e + hi_row>(r.w);
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const unsigned u = (u2 >> (16 * hh)) & 0xFFFFu;
+                    const int code = signed_code(B, u);
+                    int rv;
+                    if constexpr (B <= 2) rv = 127 * code;
+                    else { rv = ctab[(g + 8 * hi_row) * L + abs(code)]; rv = code < 0 ? -rv : rv; }
+                    packed |= ((uint32_t)rv & 0xFFu) << (8 * (2 * e + hh));
+                }
+            });
+            A[rr] = packed;
+        });
+#pragma unroll
+        for (int tb = 0; tb < NT; ++tb) {
+            const uint32_t b0 = *(const uint32_t *)(xl + tb * 8 * XS + 16 * j);
+            const uint32_t b1 = *(const uint32_t *)(xl + tb * 8 * XS + 16 * (j + 1));
+            mma_s8(D[tb], A, b0, b1);
+        }
+    });
+    const float s_lo = __uint_as_float(p_lo.x & 0x7FFFFFFFu), s_hi = __uint_as_float(p_hi.x & 0x7FFFFFFFu);
+#pragma unroll
+    for (int tb = 0; tb < NT; ++tb) {
+        acc[tb][0] = fmaf(s_lo, (float)D[tb][0], acc[tb][0]);
+        acc[tb][1] = fmaf(s_lo, (float)D[tb][1], acc[tb][1]);
+        acc[tb][2] = fmaf(s_hi, (float)D[tb][2], acc[tb][2]);
+        acc[tb][3] = fmaf(s_hi, (float)D[tb][3], acc[tb][3]);
+    }
+}
+
+template <int B, int G, int NT, int MODE>
+__device__ __forceinline__ void compute_tile(const TileRegs<B, TILE / G> &r, const uint8_t *xl, int XS, int8_t *ctab,
+                                             int g, int t, float (&acc)[NT][4]) {
+    constexpr int GPT = TILE / G;
+    static_for<GPT>([&](auto gc) {
+        constexpr int GI = decltype(gc)::value;
+        if constexpr (MODE == 0) {
+            const bool fix = B > 1 && __any_sync(0xffffffffu, (r.prm[0][GI].x | r.prm[1][GI].x) >> 31);
+            if (!fix) group_model<B, G, NT, GI, false>(r, reinterpret_cast<const __half *>(xl), XS, acc);
+            else group_model<B, G, NT, GI, true>(r, reinterpret_cast<const __half *>(xl), XS, acc);
+        } else {
+            group_a8<B, G, NT, GI>(r, reinterpret_cast<const int8_t *>(xl), XS, ctab, g, t, acc);
+        }
+    });
+}
+
+// CTA index that owns linear tile `tile` when T tiles are cut into P runs [floor(c T / P), floor((c+1) T / P)).
+__host__ __device__ inline int owner_of(int64_t tile, int64_t T, int64_t P) { return (int)(((tile + 1) * P - 1) / T); }
 
 // ------------------------------------------------------------------------------------------
 // MODE 0: model dtype.  MODE 1: Dynamic A8 (xq = int8 carrier [M][x8_pitch], dxs = row scales).
 template <int B, int G, int NT, int MODE>
-__global__ void __launch_bounds__(GEMV_THREADS)
+__global__ void __launch_bounds__(GEMV_THREADS, (NT == 1 && B <= 4 && G >= 64) ? 3 : 2)
 gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restrict__ x, const int8_t *__restrict__ xq,
-            int64_t x8_pitch, const float *__restrict__ dxs, uint16_t *__restrict__ y, int M, int S,
+            int64_t x8_pitch, const float *__restrict__ dxs, uint16_t *__restrict__ y, int M, int max_slots,
             float *__restrict__ partial, int *__restrict__ counters) {
-    constexpr int GPT = TILE / G;      // groups per tile
-    constexpr int CPG = G / 16;        // 16-wide k chunks per group
+    constexpr int GPT = TILE / G;
     constexpr int L = B == 1 ? 1 : (1 << (B - 1));
+    constexpr int RT = 8 * NT;       // staged token rows (rows >= M are zero)
+    constexpr int NBUF = (B <= 4) ? 3 : 2;
+    constexpr int ES = MODE == 0 ? 2 : 1;  // bytes per staged activation element
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ float s_inv[16];
     __shared__ unsigned s_max[16];
     __shared__ int s_last;
 
-    const int nb = blockIdx.x / S, sk = blockIdx.x % S;
-    const int kb0 = (int)(((int64_t)sk * d.KT) / S), kb1 = (int)(((int64_t)(sk + 1) * d.KT) / S);
-    const int slice_k = (kb1 - kb0) * TILE;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    const int64_t k_base = (int64_t)kb0 * TILE;
-
-    const uint8_t *tile0 = layout + ((size_t)nb * d.KT + kb0) * (size_t)d.tile_bytes;
-    const uint8_t *rbp0 = tile0 + warp * 256 * B;
-    const uint8_t *prm0 = tile0 + d.code_bytes + ((warp * 16 + g) * GPT) * 8;  // row g of this row block
-
-    // issue the first weight loads before touching the activations
-    constexpr int PF = (B <= 4) ? 2 : 1;
-    Rec<B> rec[PF + 1];
-    GroupParams prm[PF + 1][2][GPT];
-#pragma unroll
-    for (int i = 0; i < PF; ++i)
-        if (kb0 + i < kb1) {
-            load_rec<B>(rec[i], rbp0 + (size_t)i * d.tile_bytes, lane);
-#pragma unroll
-            for (int gi = 0; gi < GPT; ++gi) {
-                prm[i][0][gi] = *(const GroupParams *)(prm0 + (size_t)i * d.tile_bytes + gi * 8);
-                prm[i][1][gi] = *(const GroupParams *)(prm0 + (size_t)i * d.tile_bytes + (8 * GPT + gi) * 8);
-            }
-        }
-
-    // ---- stage the activation slice
-    const int XS = slice_k + XS_PAD;  // elements per staged row
-    if constexpr (MODE == 0) {
-        __half *xs = reinterpret_cast<__half *>(smem);
-        if (threadIdx.x < 16) s_max[threadIdx.x] = 0;
-        __syncthreads();
-        const int cpr = slice_k / 8;  // 16-byte chunks per row
-        const bool vec = (d.K % 8) == 0;
-        for (int idx = threadIdx.x; idx < M * cpr; idx += GEMV_THREADS) {
-            const int m = idx / cpr, c = idx % cpr;
-            const int64_t k = k_base + (int64_t)c * 8;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (vec) {
-                if (k < d.K) v = *(const uint4 *)(x + (int64_t)m * d.K + k);
-            } else {
-                uint16_t e[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) e[q] = (k + q < d.K) ? x[(int64_t)m * d.K + k + q] : (uint16_t)0;
-                v.x = e[0] | (e[1] << 16); v.y = e[2] | (e[3] << 16); v.z = e[4] | (e[5] << 16); v.w = e[6] | (e[7] << 16);
-            }
-            *(uint4 *)(xs + m * XS + c * 8) = v;  // raw bf16 for now
-            unsigned mx = 0;  // largest |bf16| bit pattern of the chunk
-            const uint32_t ws[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int q = 0; q < 4; ++q) { mx = max(mx, ws[q] & 0x7FFFu); mx = max(mx, (ws[q] >> 16) & 0x7FFFu); }
-            atomicMax(&s_max[m], mx);
-        }
-        __syncthreads();
-        if (threadIdx.x < 16) {
-            // power-of-two scale putting the row maximum in [2^14, 2^15)
-            const float mxf = __uint_as_float(s_max[threadIdx.x] << 16);
-            int sh = 0;
-            if (mxf > 0.0f && mxf < 3.0e38f) sh = 14 - (int)((s_max[threadIdx.x] >> 7) & 0xFF) + 127;
-            sh = max(min(sh, 100), -100);
-            s_inv[threadIdx.x] = exp2f((float)(-sh));
-        }
-        __syncthreads();
-        for (int idx = threadIdx.x; idx < M * cpr; idx += GEMV_THREADS) {
-            const int m = idx / cpr, c = idx % cpr;
-            const float sc = 1.0f / s_inv[m];
-            uint4 v = *(uint4 *)(xs + m * XS + c * 8);
-            uint32_t ws[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const float lo = __uint_as_float(ws[q] << 16) * sc, hi = __uint_as_float(ws[q] & 0xFFFF0000u) * sc;
-                const __half2 h = __floats2half2_rn(lo, hi);
-                ws[q] = *reinterpret_cast<const uint32_t *>(&h);
-            }
-            *(uint4 *)(xs + m * XS + c * 8) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
-        }
-    } else {
-        int8_t *xs = reinterpret_cast<int8_t *>(smem);
-        const int cpr = slice_k / 16;
-        for (int idx = threadIdx.x; idx < M * cpr; idx += GEMV_THREADS) {
-            const int m = idx / cpr, c = idx % cpr;
-            // the carrier is written with a pitch that is a multiple of 128, zero beyond K
-            *(uint4 *)(xs + m * XS + c * 16) = *(const uint4 *)(xq + (int64_t)m * x8_pitch + k_base + c * 16);
-        }
-        if (threadIdx.x < 16) s_inv[threadIdx.x] = threadIdx.x < M ? dxs[threadIdx.x] * (1.0f / 127.0f) : 0.0f;
-    }
-    __syncthreads();
-
-    // per-warp carrier table (A8): [16 rows][L] int8 after the activation rows
+    const int64_t T = (int64_t)d.NB * d.KT, P = gridDim.x;
+    const int64_t t_begin = ((int64_t)blockIdx.x * T) / P, t_end = ((int64_t)(blockIdx.x + 1) * T) / P;
     int8_t *ctab = nullptr;
-    if constexpr (MODE == 1 && B >= 3) ctab = reinterpret_cast<int8_t *>(smem) + 16 * XS + warp * 16 * L;
+    if constexpr (MODE == 1 && B >= 3) ctab = reinterpret_cast<int8_t *>(smem) + RT * (MAX_SUB * TILE + XS_PAD) + warp * 16 * L;
 
-    float acc[NT][4];
+    for (int64_t tile = t_begin; tile < t_end;) {
+        const int nb = (int)(tile / d.KT), kb_begin = (int)(tile % d.KT);
+        const int kb_end = (int)min((int64_t)d.KT, kb_begin + (t_end - tile));
+        float total[NT][4];
 #pragma unroll
-    for (int tb = 0; tb < NT; ++tb)
+        for (int tb = 0; tb < NT; ++tb)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) acc[tb][i] = 0.0f;
+            for (int i = 0; i < 4; ++i) total[tb][i] = 0.0f;
 
-    for (int kb = kb0; kb < kb1; ++kb) {
-        // prefetch PF tiles ahead
-        if (kb + PF < kb1) {
-            const size_t off = (size_t)(kb + PF - kb0) * d.tile_bytes;
-            load_rec<B>(rec[PF], rbp0 + off, lane);
-#pragma unroll
-            for (int gi = 0; gi < GPT; ++gi) {
-                prm[PF][0][gi] = *(const GroupParams *)(prm0 + off + gi * 8);
-                prm[PF][1][gi] = *(const GroupParams *)(prm0 + off + (8 * GPT + gi) * 8);
-            }
-        }
-        const int kl = (kb - kb0) * TILE;  // k offset inside the staged slice
-#pragma unroll
-        for (int gi = 0; gi < GPT; ++gi) {
-            const GroupParams p_lo = prm[0][0][gi], p_hi = prm[0][1][gi];
-            const bool fix = B > 1 && __any_sync(0xffffffffu, (__float_as_uint(p_lo.s) | __float_as_uint(p_hi.s)) >> 31);
+        for (int ks = kb_begin; ks < kb_end; ks += MAX_SUB) {
+            const int ke = min(kb_end, ks + MAX_SUB);
+            const int slice_k = (ke - ks) * TILE, XS = slice_k + XS_PAD;
+            const int64_t k_base = (int64_t)ks * TILE;
+            const uint8_t *tile0 = layout + ((size_t)nb * d.KT + ks) * (size_t)d.tile_bytes;
+            const uint8_t *rbp0 = tile0 + warp * 256 * B;
+            const uint8_t *prm0 = tile0 + d.code_bytes + ((warp * 16 + g) * GPT) * 8;
+
+            // first weight loads go out before the activations are touched
+            TileRegs<B, GPT> buf[NBUF];
+            static_for<NBUF>([&](auto ic) {
+                constexpr int i = decltype(ic)::value;
+                if (ks + i < ke) load_tile<B, GPT>(buf[i], rbp0 + (size_t)i * d.tile_bytes, prm0 + (size_t)i * d.tile_bytes, lane);
+            });
+
+            // ---- stage the activation slice [k_base, k_base + slice_k) for RT token rows
+            __syncthreads();  // previous slice fully consumed
             if constexpr (MODE == 0) {
-                const RowCoef c_lo = make_coef<B>(p_lo), c_hi = make_coef<B>(p_hi);
-                float D[NT][4];
+                __half *xs = reinterpret_cast<__half *>(smem);
+                if (threadIdx.x < 16) s_max[threadIdx.x] = 0;
+                __syncthreads();
+                const int cpr = slice_k / 8;  // 16-byte chunks per row
+                for (int idx = threadIdx.x; idx < RT * cpr; idx += GEMV_THREADS) {
+                    const int m = idx / cpr, c = idx % cpr;
+                    const int64_t k = k_base + (int64_t)c * 8;
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (m < M && k < d.K) v = *(const uint4 *)(x + (int64_t)m * d.K + k);  // K % 8 == 0 always
+                    *(uint4 *)(xs + m * XS + c * 8) = v;  // raw bf16 for now
+                    if (m < M) {
+                        unsigned mx = 0;  // largest |bf16| bit pattern of the chunk
+                        const uint32_t ws[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-                for (int tb = 0; tb < NT; ++tb)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) D[tb][i] = 0.0f;
-                const __half *xs = reinterpret_cast<const __half *>(smem);
-#pragma unroll
-                for (int jj = 0; jj < CPG; ++jj) {
-                    const int j = gi * CPG + jj;
-                    uint32_t A[4];
-                    if (!fix) {
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) A[i] = level_pair<B, false>(pair_T<B>(rec[0].w, 4 * j + i), (i & 1) ? c_hi : c_lo);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) A[i] = level_pair<B, true>(pair_T<B>(rec[0].w, 4 * j + i), (i & 1) ? c_hi : c_lo);
-                    }
-#pragma unroll
-                    for (int tb = 0; tb < NT; ++tb) {
-                        const int tok = tb * 8 + g;
-                        uint2 bf = make_uint2(0, 0);
-                        if (tok < M) bf = *(const uint2 *)(xs + tok * XS + kl + 16 * j + 4 * t);
-                        mma_f16(D[tb], A, bf.x, bf.y);
+                        for (int q = 0; q < 4; ++q) { mx = max(mx, ws[q] & 0x7FFFu); mx = max(mx, (ws[q] >> 16) & 0x7FFFu); }
+                        if (mx) atomicMax(&s_max[m], mx);
                     }
                 }
+                __syncthreads();
+                if (threadIdx.x < 16) {
+                    // power-of-two scale putting the row maximum in [2^14, 2^15)
+                    const unsigned mb = s_max[threadIdx.x];
+                    const float mxf = __uint_as_float(mb << 16);
+                    int sh = 0;
+                    if (mxf > 0.0f && mxf < 3.0e38f) sh = 14 - (int)((mb >> 7) & 0xFF) + 127;
+                    sh = max(min(sh, 100), -100);
+                    s_inv[threadIdx.x] = exp2f((float)(-sh));
+                }
+                __syncthreads();
+                for (int idx = threadIdx.x; idx < M * cpr; idx += GEMV_THREADS) {
+                    const int m = idx / cpr, c = idx % cpr;
+                    const float sc = 1.0f / s_inv[m];
+                    uint4 v = *(uint4 *)(xs + m * XS + c * 8);
+                    uint32_t ws[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-                for (int tb = 0; tb < NT; ++tb) {
-                    acc[tb][0] = fmaf(c_lo.s, D[tb][0], acc[tb][0]);
-                    acc[tb][1] = fmaf(c_lo.s, D[tb][1], acc[tb][1]);
-                    acc[tb][2] = fmaf(c_hi.s, D[tb][2], acc[tb][2]);
-                    acc[tb][3] = fmaf(c_hi.s, D[tb][3], acc[tb][3]);
+                    for (int q = 0; q < 4; ++q) {
+                        const float lo = __uint_as_float(ws[q] << 16) * sc, hi = __uint_as_float(ws[q] & 0xFFFF0000u) * sc;
+                        ws[q] = as_u32(__floats2half2_rn(lo, hi));
+                    }
+                    *(uint4 *)(xs + m * XS + c * 8) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
                 }
             } else {
-                // carrier table of this group for the warp's 16 rows: lane (g, t) fills entries i = t mod 4
-                if constexpr (B >= 3) {
-                    __syncwarp();
-                    const float a_lo = __half2float(p_lo.a), b_lo = __half2float(p_lo.b);
-                    const float a_hi = __half2float(p_hi.a), b_hi = __half2float(p_hi.b);
-                    for (int i = t; i < L; i += 4) {
-                        ctab[g * L + i] = (int8_t)carrier_of(B, i, a_lo, b_lo);
-                        ctab[(g + 8) * L + i] = (int8_t)carrier_of(B, i, a_hi, b_hi);
-                    }
-                    __syncwarp();
+                int8_t *xs = reinterpret_cast<int8_t *>(smem);
+                const int cpr = slice_k / 16;
+                for (int idx = threadIdx.x; idx < RT * cpr; idx += GEMV_THREADS) {
+                    const int m = idx / cpr, c = idx % cpr;
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    // the carrier has a pitch that is a multiple of 128 and is zero beyond K
+                    if (m < M) v = *(const uint4 *)(xq + (int64_t)m * x8_pitch + k_base + c * 16);
+                    *(uint4 *)(xs + m * XS + c * 16) = v;
                 }
-                int D[NT][4];
+                if (threadIdx.x < 16) s_inv[threadIdx.x] = threadIdx.x < M ? dxs[threadIdx.x] * (1.0f / 127.0f) : 0.0f;
+            }
+            __syncthreads();
+
+            // ---- stream the tiles of this slice
+            float acc[NT][4];
 #pragma unroll
-                for (int tb = 0; tb < NT; ++tb)
+            for (int tb = 0; tb < NT; ++tb)
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) D[tb][i] = 0;
-                const int8_t *xs = reinterpret_cast<const int8_t *>(smem);
-#pragma unroll
-                for (int jj = 0; jj < CPG; jj += 2) {
-                    const int j = gi * CPG + jj;
-                    uint32_t A[4];
-                    // a0: row g chunk j; a1: row g+8 chunk j; a2: row g chunk j+1; a3: row g+8 chunk j+1
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) {
-                        const int jc = j + (r >> 1), hi_row = r & 1;
-                        uint32_t packed = 0;
-#pragma unroll
-                        for (int e = 0; e < 2; ++e) {  // registers (hi_row) and (2 + hi_row) hold k+0,1 and k+2,3
-                            const uint32_t u2 = pair_codes<B>(rec[0].w, 4 * jc + 2 * e + hi_row);
-#pragma unroll
-                            for (int hh = 0; hh < 2; ++hh) {
-                                const unsigned u = (u2 >> (16 * hh)) & 0xFFFFu;
-                                const int code = signed_code(B, u);
-                                int rv;
-                                if constexpr (B <= 2) rv = 127 * code;
-                                else { rv = ctab[(g + 8 * hi_row) * L + abs(code)]; rv = code < 0 ? -rv : rv; }
-                                packed |= ((uint32_t)rv & 0xFFu) << (8 * (2 * e + hh));
-                            }
+                for (int i = 0; i < 4; ++i) acc[tb][i] = 0.0f;
+            const uint8_t *xlane = smem + (size_t)(g * XS + 4 * t) * ES;
+            for (int kb = ks; kb < ke; kb += NBUF) {
+                static_for<NBUF>([&](auto ic) {
+                    constexpr int i = decltype(ic)::value;
+                    if (kb + i < ke) {
+                        compute_tile<B, G, NT, MODE>(buf[i], xlane + (size_t)(kb + i - ks) * TILE * ES, XS, ctab, g, t, acc);
+                        if (kb + i + NBUF < ke) {
+                            const size_t off = (size_t)(kb + i + NBUF - ks) * d.tile_bytes;
+                            load_tile<B, GPT>(buf[i], rbp0 + off, prm0 + off, lane);
                         }
-                        A[r] = packed;
                     }
+                });
+            }
+            // fold the slice in true units: lane (g, t) holds rows g, g+8 x tokens 2t, 2t+1
 #pragma unroll
-                    for (int tb = 0; tb < NT; ++tb) {
-                        const int tok = tb * 8 + g;
-                        uint32_t b0 = 0, b1 = 0;
-                        if (tok < M) {
-                            b0 = *(const uint32_t *)(xs + tok * XS + kl + 16 * j + 4 * t);
-                            b1 = *(const uint32_t *)(xs + tok * XS + kl + 16 * (j + 1) + 4 * t);
-                        }
-                        mma_s8(D[tb], A, b0, b1);
-                    }
-                }
-                const float s_lo = fabsf(p_lo.s), s_hi = fabsf(p_hi.s);
+            for (int tb = 0; tb < NT; ++tb)
 #pragma unroll
-                for (int tb = 0; tb < NT; ++tb) {
-                    acc[tb][0] = fmaf(s_lo, (float)D[tb][0], acc[tb][0]);
-                    acc[tb][1] = fmaf(s_lo, (float)D[tb][1], acc[tb][1]);
-                    acc[tb][2] = fmaf(s_hi, (float)D[tb][2], acc[tb][2]);
-                    acc[tb][3] = fmaf(s_hi, (float)D[tb][3], acc[tb][3]);
+                for (int i = 0; i < 4; ++i) total[tb][i] = fmaf(acc[tb][i], s_inv[tb * 8 + 2 * t + (i & 1)], total[tb][i]);
+        }
+
+        // ---- finish this row block
+        const bool whole = (kb_begin == 0 && kb_end == d.KT);
+        const int c_first = owner_of((int64_t)nb * d.KT, T, P);
+        const int n_contrib = owner_of((int64_t)(nb + 1) * d.KT - 1, T, P) - c_first + 1;
+        const int slot = (int)blockIdx.x - c_first;
+        const int64_t n_lo = (int64_t)nb * TILE + warp * 16 + g;
+        float *pslot = partial + ((size_t)nb * max_slots + slot) * (size_t)(M * TILE);
+#pragma unroll
+        for (int tb = 0; tb < NT; ++tb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int tok = tb * 8 + 2 * t + (i & 1);
+                const int r = warp * 16 + g + ((i >> 1) ? 8 : 0);
+                if (tok >= M) continue;
+                if (whole) {
+                    const int64_t n = n_lo + ((i >> 1) ? 8 : 0);
+                    if (n < d.N) y[(int64_t)tok * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(total[tb][i]));
+                } else {
+                    pslot[tok * TILE + r] = total[tb][i];
                 }
             }
-        }
-        // rotate the prefetch registers
-#pragma unroll
-        for (int i = 0; i < PF; ++i) {
-            rec[i] = rec[i + 1];
-#pragma unroll
-            for (int gi = 0; gi < GPT; ++gi) { prm[i][0][gi] = prm[i + 1][0][gi]; prm[i][1][gi] = prm[i + 1][1][gi]; }
-        }
-    }
-
-    // ---- epilogue: lane (g, t) holds rows g, g+8 x tokens 2t, 2t+1 of each token block
-    const int64_t Np = (int64_t)d.NB * TILE;
-    const int64_t n_lo = (int64_t)nb * TILE + warp * 16 + g;
-#pragma unroll
-    for (int tb = 0; tb < NT; ++tb)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int tok = tb * 8 + 2 * t + (i & 1);
-            const int64_t n = n_lo + ((i >> 1) ? 8 : 0);
-            if (tok >= M) continue;
-            const float v = acc[tb][i] * s_inv[tok];
-            if (S == 1) {
-                if (n < d.N) y[(int64_t)tok * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
-            } else {
-                partial[((int64_t)sk * M + tok) * Np + n] = v;
+        if (!whole) {
+            // the last CTA to arrive at this row block adds the slots in slot order
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) s_last = (atomicAdd(&counters[nb], 1) == n_contrib - 1);
+            __syncthreads();
+            if (s_last) {
+                __threadfence();
+                const float *pb = partial + (size_t)nb * max_slots * (size_t)(M * TILE);
+                for (int idx = threadIdx.x; idx < M * TILE; idx += GEMV_THREADS) {
+                    const int m = idx / TILE, r = idx % TILE;
+                    const int64_t n = (int64_t)nb * TILE + r;
+                    float sum = 0.0f;
+                    for (int q = 0; q < n_contrib; ++q) sum += __ldcg(pb + (size_t)q * (M * TILE) + idx);
+                    if (n < d.N) y[(int64_t)m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(sum));
+                }
+                if (threadIdx.x == 0) counters[nb] = 0;  // leave the workspace ready for the next call
             }
         }
-    if (S == 1) return;
-
-    // ---- split-K combine: the last CTA of this row block to arrive sums the slices in index order
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const int old = atomicAdd(&counters[nb], 1);
-        s_last = (old == S - 1);
+        tile += (kb_end - kb_begin);
     }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    for (int idx = threadIdx.x; idx < M * TILE; idx += GEMV_THREADS) {
-        const int m = idx / TILE, r = idx % TILE;
-        const int64_t n = (int64_t)nb * TILE + r;
-        float sum = 0.0f;
-        for (int q = 0; q < S; ++q) sum += __ldcg(&partial[((int64_t)q * M + m) * Np + n]);
-        if (n < d.N) y[(int64_t)m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(sum));
-    }
-    if (threadIdx.x == 0) counters[nb] = 0;  // leave the workspace ready for the next call
 }
 
 template <int B, int G, int NT, int MODE>
 cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, const int8_t *xq, int64_t x8_pitch,
-                       const float *dxs, uint16_t *y, int M, int S, float *partial, int *counters, cudaStream_t st) {
-    const int slice_tiles = (d.KT + S - 1) / S;
-    const int XS = slice_tiles * TILE + XS_PAD;
-    size_t smem = MODE == 0 ? (size_t)M * XS * 2 : (size_t)16 * XS + 8 * 16 * (B == 1 ? 1 : (1 << (B - 1)));
+                       const float *dxs, uint16_t *y, int M, int P, int max_slots, float *partial, int *counters,
+                       cudaStream_t st) {
+    constexpr int RT = 8 * NT;
+    constexpr int L = B == 1 ? 1 : (1 << (B - 1));
+    const int64_t T = (int64_t)d.NB * d.KT;
+    int64_t sub64 = (T + P - 1) / P + 1;
+    if (sub64 > d.KT) sub64 = d.KT;
+    if (sub64 > MAX_SUB) sub64 = MAX_SUB;
+    const int sub_tiles = (int)sub64;
+    const int XS = sub_tiles * TILE + XS_PAD;
+    size_t smem = MODE == 0 ? (size_t)RT * XS * 2 : (size_t)RT * (MAX_SUB * TILE + XS_PAD) + 8 * 16 * L;
     auto kern = gemv_kernel<B, G, NT, MODE>;
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static bool attr_done = false;
+    if (smem > 48 * 1024 && !attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
         if (e != cudaSuccess) return e;
+        attr_done = true;
     }
-    kern<<<d.NB * S, GEMV_THREADS, smem, st>>>((const uint8_t *)layout, d, x, xq, x8_pitch, dxs, y, M, S, partial, counters);
+    kern<<<P, GEMV_THREADS, smem, st>>>((const uint8_t *)layout, d, x, xq, x8_pitch, dxs, y, M, max_slots, partial, counters);
     return cudaGetLastError();
 }
 
 template <int B, int G>
 cudaError_t dispatch_nt_mode(const void *layout, const Dims &d, const uint16_t *x, const int8_t *xq, int64_t x8_pitch,
-                             const float *dxs, uint16_t *y, int M, int mode, int S, float *partial, int *counters,
-                             cudaStream_t st) {
+                             const float *dxs, uint16_t *y, int M, int mode, int P, int max_slots, float *partial,
+                             int *counters, cudaStream_t st) {
     if (mode == 0) {
-        if (M <= 8) return launch_one<B, G, 1, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, S, partial, counters, st);
-        return launch_one<B, G, 2, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, S, partial, counters, st);
+        if (M <= 8) return launch_one<B, G, 1, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, partial, counters, st);
+        return launch_one<B, G, 2, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, partial, counters, st);
     }
-    if (M <= 8) return launch_one<B, G, 1, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, S, partial, counters, st);
-    return launch_one<B, G, 2, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, S, partial, counters, st);
+    if (M <= 8) return launch_one<B, G, 1, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, partial, counters, st);
+    return launch_one<B, G, 2, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, partial, counters, st);
 }
 
 template <int B>
 cudaError_t dispatch_g(const void *layout, const Dims &d, const uint16_t *x, const int8_t *xq, int64_t x8_pitch,
-                       const float *dxs, uint16_t *y, int M, int mode, int S, float *partial, int *counters,
-                       cudaStream_t st) {
+                       const float *dxs, uint16_t *y, int M, int mode, int P, int max_slots, float *partial,
+                       int *counters, cudaStream_t st) {
     switch (d.G) {
-        case 32: return dispatch_nt_mode<B, 32>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, S, partial, counters, st);
-        case 64: return dispatch_nt_mode<B, 64>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, S, partial, counters, st);
-        default: return dispatch_nt_mode<B, 128>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, S, partial, counters, st);
+        case 32: return dispatch_nt_mode<B, 32>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_slots, partial, counters, st);
+        case 64: return dispatch_nt_mode<B, 64>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_slots, partial, counters, st);
+        default: return dispatch_nt_mode<B, 128>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_slots, partial, counters, st);
     }
 }
 
 }  // namespace
 
-// Split-K factor of the small-M path: enough CTAs to fill 148 SMs about three times over, at
-// most MAX_SLICE_TILES K tiles per CTA, at least one.
-int gemv_split_k(const Dims &d) {
-    int S = (444 + d.NB - 1) / d.NB;
-    if (S > d.KT) S = d.KT;
-    const int min_s = (d.KT + MAX_SLICE_TILES - 1) / MAX_SLICE_TILES;
-    if (S < min_s) S = min_s;
-    if (S < 1) S = 1;
-    return S;
+// Number of CTAs of the small-M path (one run of tiles each) and the most CTAs that can
+// contribute to one row block.  148 SMs x 3 resident CTAs for M <= 8, B <= 4 and G >= 64, x 2 otherwise
+// (matches the __launch_bounds__ of the kernel).
+GemvPlan gemv_plan(const Dims &d, int64_t M) {
+    GemvPlan p;
+    const int64_t T = (int64_t)d.NB * d.KT;
+    int64_t P = (M <= 8 && d.B <= 4 && d.G >= 64) ? 148 * 3 : 148 * 2;
+    if (P > T) P = T;
+    p.ctas = (int)P;
+    int mx = 1;
+    for (int nb = 0; nb < d.NB; ++nb) {
+        const int c = owner_of((int64_t)(nb + 1) * d.KT - 1, T, P) - owner_of((int64_t)nb * d.KT, T, P) + 1;
+        if (c > mx) mx = c;
+    }
+    p.max_slots = mx;
+    return p;
 }
 
 cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
                         uint8_t *ws, const Workspace &plan, cudaStream_t st) {
-    const int S = plan.split_k;
+    const GemvPlan gp = gemv_plan(d, M);
     float *partial = reinterpret_cast<float *>(ws + plan.partial_off);
     int *counters = reinterpret_cast<int *>(ws + plan.counters_off);
     int8_t *xq = reinterpret_cast<int8_t *>(ws + plan.x8_off);
@@ -476,15 +539,16 @@ cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, ui
         cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, st);
         if (e != cudaSuccess) return e;
     }
+    const int Mi = (int)M, P = gp.ctas, ms = gp.max_slots;
     switch (d.B) {
-        case 1: return dispatch_g<1>(layout, d, x, xq, pitch, dxs, y, (int)M, mode, S, partial, counters, st);
-        case 2: return dispatch_g<2>(layout, d, x, xq, pitch, dxs, y, (int)M, mode, S, partial, counters, st);
-        case 3: return dispatch_g<3>(layout, d, x, xq, pitch, dxs, y, (int)M, mode, S, partial, counters, st);
-        case 4: return dispatch_g<4>(layout, d, x, xq, pitch, dxs, y, (int)M, mode, S, partial, counters, st);
-        case 5: return dispatch_g<5>(layout, d, x, xq, pitch, dxs, y, (int)M, mode, S, partial, counters, st);
-        case 6: return dispatch_g<6>(layout, d, x, xq, pitch, dxs, y, (int)M, mode, S, partial, counters, st);
-        case 7: return dispatch_g<7>(layout, d, x, xq, pitch, dxs, y, (int)M, mode, S, partial, counters, st);
-        default: return dispatch_g<8>(layout, d, x, xq, pitch, dxs, y, (int)M, mode, S, partial, counters, st);
+        case 1: return dispatch_g<1>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
+        case 2: return dispatch_g<2>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
+        case 3: return dispatch_g<3>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
+        case 4: return dispatch_g<4>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
+        case 5: return dispatch_g<5>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
+        case 6: return dispatch_g<6>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
+        case 7: return dispatch_g<7>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
+        default: return dispatch_g<8>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
     }
 }
 

@@ -22,14 +22,18 @@ cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *
 // Workspace carving (all offsets 256-byte aligned).
 struct Workspace {
     size_t counters_off, counters_bytes;   // int32 arrival counters, one per 128-row block
-    size_t partial_off, partial_bytes;     // fp32 split-K partial sums [S][M][Np]
+    size_t partial_off, partial_bytes;     // fp32 split-K partial sums [NB][max_slots][M][128]
     size_t x8_off, x8_bytes;               // Dynamic A8: int8 activation carrier [M][Kp]
     size_t dx_off, dx_bytes;               // Dynamic A8: row scales [M]
     size_t status_off;                     // int32 device status word (bounded waits report here)
     size_t total;
-    int split_k;                           // S used by the small-M path
 };
 Workspace plan_workspace(const Dims &d, int64_t M, int mode);
+
+// Decomposition of the small-M path: number of CTAs (one contiguous run of tiles each) and the
+// largest number of CTAs that contribute to one 128-row block.
+struct GemvPlan { int ctas, max_slots; };
+GemvPlan gemv_plan(const Dims &d, int64_t M);
 
 // Small-M (M <= 16) split-K tensor-core GEMV, both activation modes.
 cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
