@@ -8,7 +8,7 @@ from dataclasses import dataclass
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libcubicquant.so")
+_LIB_PATH = os.environ.get("CUBICQUANT_LIB") or os.path.join(_HERE, "libcubicquant.so")
 
 CQ_MODEL_DTYPE = 0
 CQ_DYN_A8 = 1

@@ -29,6 +29,9 @@ namespace {
 constexpr int GEMV_THREADS = 256;
 constexpr int XS_PAD = 16;     // elements of padding per staged activation row (bank spread)
 constexpr int MAX_SUB = 16;    // K tiles staged at a time (bounds shared memory)
+#ifndef CQ_GEMV_OCC_HI
+#define CQ_GEMV_OCC_HI 3       // resident CTAs per SM asked of the compiler for the light variants
+#endif
 
 template <int... I, class F>
 __device__ __forceinline__ void static_for_impl(F &&f, std::integer_sequence<int, I...>) {
@@ -40,13 +43,13 @@ __device__ __forceinline__ void static_for(F &&f) {
 }
 
 __device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
+    asm(
         "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ void mma_s8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
+    asm(
         "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
         : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
@@ -54,12 +57,12 @@ __device__ __forceinline__ void mma_s8(int (&d)[4], const uint32_t (&a)[4], uint
 
 __device__ __forceinline__ uint4 ld_stream16(const void *p) {
     uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    asm("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
 }
 __device__ __forceinline__ uint2 ld_stream8(const void *p) {
     uint2 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    asm("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
     return v;
 }
 
@@ -78,22 +81,23 @@ struct TileRegs {
     uint2 prm[2][GPT];  // {s bits, a | b << 16} of rows g and g + 8
 };
 
+// wl = row-block base + lane * 16 (codes); pl = parameter record of row g of the row block.
 template <int B, int GPT>
-__device__ __forceinline__ void load_tile(TileRegs<B, GPT> &r, const uint8_t *rbp, const uint8_t *prm, int lane) {
+__device__ __forceinline__ void load_tile(TileRegs<B, GPT> &r, const uint8_t *wl, const uint8_t *pl, int lane) {
     constexpr int NFQ = (2 * B) / 4;
 #pragma unroll
     for (int q = 0; q < NFQ; ++q) {
-        const uint4 v = ld_stream16(rbp + (q * 32 + lane) * 16);
+        const uint4 v = ld_stream16(wl + q * 512);
         r.w[4 * q + 0] = v.x; r.w[4 * q + 1] = v.y; r.w[4 * q + 2] = v.z; r.w[4 * q + 3] = v.w;
     }
     if constexpr ((2 * B) % 4 != 0) {
-        const uint2 v = ld_stream8(rbp + NFQ * 512 + lane * 8);
+        const uint2 v = ld_stream8(wl + NFQ * 512 - lane * 8);  // the tail is indexed lane * 8, not lane * 16
         r.w[4 * NFQ + 0] = v.x; r.w[4 * NFQ + 1] = v.y;
     }
 #pragma unroll
     for (int gi = 0; gi < GPT; ++gi) {
-        r.prm[0][gi] = ld_stream8(prm + gi * 8);
-        r.prm[1][gi] = ld_stream8(prm + (8 * GPT + gi) * 8);
+        r.prm[0][gi] = ld_stream8(pl + gi * 8);
+        r.prm[1][gi] = ld_stream8(pl + (8 * GPT + gi) * 8);
     }
 }
 
@@ -177,11 +181,14 @@ template <int B, int G, int NT, int GI, bool FIX>
 __device__ __forceinline__ void group_model(const TileRegs<B, TILE / G> &r, const __half *xl, int XS, float (&acc)[NT][4]) {
     constexpr int CPG = G / 16;
     const RowCoef c_lo = make_coef<B>(r.prm[0][GI]), c_hi = make_coef<B>(r.prm[1][GI]);
-    float D[NT][4];
+    // two accumulator sets so consecutive MMAs do not wait on each other
+    float D[2][NT][4];
 #pragma unroll
-    for (int tb = 0; tb < NT; ++tb)
+    for (int h = 0; h < 2; ++h)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) D[tb][i] = 0.0f;
+        for (int tb = 0; tb < NT; ++tb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) D[h][tb][i] = 0.0f;
     static_for<CPG>([&](auto jc) {
         constexpr int j = GI * CPG + decltype(jc)::value;
         uint32_t A[4];
@@ -192,15 +199,15 @@ __device__ __forceinline__ void group_model(const TileRegs<B, TILE / G> &r, cons
 #pragma unroll
         for (int tb = 0; tb < NT; ++tb) {
             const uint2 bf = *(const uint2 *)(xl + tb * 8 * XS + 16 * j);
-            mma_f16(D[tb], A, bf.x, bf.y);
+            mma_f16(D[j & 1][tb], A, bf.x, bf.y);
         }
     });
 #pragma unroll
     for (int tb = 0; tb < NT; ++tb) {
-        acc[tb][0] = fmaf(c_lo.s, D[tb][0], acc[tb][0]);
-        acc[tb][1] = fmaf(c_lo.s, D[tb][1], acc[tb][1]);
-        acc[tb][2] = fmaf(c_hi.s, D[tb][2], acc[tb][2]);
-        acc[tb][3] = fmaf(c_hi.s, D[tb][3], acc[tb][3]);
+        acc[tb][0] = fmaf(c_lo.s, D[0][tb][0] + D[1][tb][0], acc[tb][0]);
+        acc[tb][1] = fmaf(c_lo.s, D[0][tb][1] + D[1][tb][1], acc[tb][1]);
+        acc[tb][2] = fmaf(c_hi.s, D[0][tb][2] + D[1][tb][2], acc[tb][2]);
+        acc[tb][3] = fmaf(c_hi.s, D[0][tb][3] + D[1][tb][3], acc[tb][3]);
     }
 }
 
@@ -288,7 +295,7 @@ __host__ __device__ inline int owner_of(int64_t tile, int64_t T, int64_t P) { re
 // ------------------------------------------------------------------------------------------
 // MODE 0: model dtype.  MODE 1: Dynamic A8 (xq = int8 carrier [M][x8_pitch], dxs = row scales).
 template <int B, int G, int NT, int MODE>
-__global__ void __launch_bounds__(GEMV_THREADS, (NT == 1 && B <= 4 && G >= 64) ? 3 : 2)
+__global__ void __launch_bounds__(GEMV_THREADS, (NT == 1 && B <= 4 && G >= 64) ? CQ_GEMV_OCC_HI : 2)
 gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restrict__ x, const int8_t *__restrict__ xq,
             int64_t x8_pitch, const float *__restrict__ dxs, uint16_t *__restrict__ y, int M, int max_slots,
             float *__restrict__ partial, int *__restrict__ counters) {
@@ -305,6 +312,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int64_t T = (int64_t)d.NB * d.KT, P = gridDim.x;
     const int64_t t_begin = ((int64_t)blockIdx.x * T) / P, t_end = ((int64_t)(blockIdx.x + 1) * T) / P;
+    if (threadIdx.x < 16) { s_max[threadIdx.x] = 0; s_inv[threadIdx.x] = 1.0f; }
     int8_t *ctab = nullptr;
     if constexpr (MODE == 1 && B >= 3) ctab = reinterpret_cast<int8_t *>(smem) + RT * (MAX_SUB * TILE + XS_PAD) + warp * 16 * L;
 
@@ -322,73 +330,76 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
             const int slice_k = (ke - ks) * TILE, XS = slice_k + XS_PAD;
             const int64_t k_base = (int64_t)ks * TILE;
             const uint8_t *tile0 = layout + ((size_t)nb * d.KT + ks) * (size_t)d.tile_bytes;
-            const uint8_t *rbp0 = tile0 + warp * 256 * B;
-            const uint8_t *prm0 = tile0 + d.code_bytes + ((warp * 16 + g) * GPT) * 8;
+            const uint8_t *wl = tile0 + warp * 256 * B + lane * 16;                     // next tile to load (codes)
+            const uint8_t *pl = tile0 + d.code_bytes + ((warp * 16 + g) * GPT) * 8;      // next tile to load (params)
 
             // first weight loads go out before the activations are touched
             TileRegs<B, GPT> buf[NBUF];
             static_for<NBUF>([&](auto ic) {
                 constexpr int i = decltype(ic)::value;
-                if (ks + i < ke) load_tile<B, GPT>(buf[i], rbp0 + (size_t)i * d.tile_bytes, prm0 + (size_t)i * d.tile_bytes, lane);
+                if (ks + i < ke) {
+                    load_tile<B, GPT>(buf[i], wl, pl, lane);
+                    wl += d.tile_bytes; pl += d.tile_bytes;
+                }
             });
 
             // ---- stage the activation slice [k_base, k_base + slice_k) for RT token rows
             __syncthreads();  // previous slice fully consumed
             if constexpr (MODE == 0) {
                 __half *xs = reinterpret_cast<__half *>(smem);
-                if (threadIdx.x < 16) s_max[threadIdx.x] = 0;
-                __syncthreads();
                 const int cpr = slice_k / 8;  // 16-byte chunks per row
-                for (int idx = threadIdx.x; idx < RT * cpr; idx += GEMV_THREADS) {
-                    const int m = idx / cpr, c = idx % cpr;
-                    const int64_t k = k_base + (int64_t)c * 8;
-                    uint4 v = make_uint4(0, 0, 0, 0);
-                    if (m < M && k < d.K) v = *(const uint4 *)(x + (int64_t)m * d.K + k);  // K % 8 == 0 always
-                    *(uint4 *)(xs + m * XS + c * 8) = v;  // raw bf16 for now
-                    if (m < M) {
-                        unsigned mx = 0;  // largest |bf16| bit pattern of the chunk
+                // pass 1: raw bf16 into shared memory, row maxima of |x| (as bf16 bit patterns) into s_max
+                for (int m = 0; m < RT; ++m) {
+                    unsigned mx = 0;
+                    for (int c = threadIdx.x; c < cpr; c += GEMV_THREADS) {
+                        const int64_t k = k_base + (int64_t)c * 8;
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        if (m < M && k < d.K) v = *(const uint4 *)(x + (int64_t)m * d.K + k);  // K % 8 == 0 always
+                        *(uint4 *)(xs + m * XS + c * 8) = v;
                         const uint32_t ws[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                         for (int q = 0; q < 4; ++q) { mx = max(mx, ws[q] & 0x7FFFu); mx = max(mx, (ws[q] >> 16) & 0x7FFFu); }
-                        if (mx) atomicMax(&s_max[m], mx);
+                    }
+                    if (m < M) {
+                        mx = __reduce_max_sync(0xffffffffu, mx);
+                        if (lane == 0 && mx) atomicMax(&s_max[m], mx);
                     }
                 }
                 __syncthreads();
-                if (threadIdx.x < 16) {
-                    // power-of-two scale putting the row maximum in [2^14, 2^15)
-                    const unsigned mb = s_max[threadIdx.x];
-                    const float mxf = __uint_as_float(mb << 16);
-                    int sh = 0;
-                    if (mxf > 0.0f && mxf < 3.0e38f) sh = 14 - (int)((mb >> 7) & 0xFF) + 127;
+                // pass 2: every thread derives the power-of-two scale that puts the row maximum in
+                // [2^14, 2^15) and converts the chunks it wrote
+                for (int m = 0; m < M; ++m) {
+                    const unsigned mb = s_max[m];
+                    const int ef = (int)((mb >> 7) & 0xFF);          // biased exponent of the maximum
+                    int sh = (mb == 0 || ef == 255) ? 0 : 14 - ef + 127;
                     sh = max(min(sh, 100), -100);
-                    s_inv[threadIdx.x] = exp2f((float)(-sh));
-                }
-                __syncthreads();
-                for (int idx = threadIdx.x; idx < M * cpr; idx += GEMV_THREADS) {
-                    const int m = idx / cpr, c = idx % cpr;
-                    const float sc = 1.0f / s_inv[m];
-                    uint4 v = *(uint4 *)(xs + m * XS + c * 8);
-                    uint32_t ws[4] = {v.x, v.y, v.z, v.w};
+                    const float sc = __uint_as_float((uint32_t)(127 + sh) << 23);   // 2^sh
+                    if (threadIdx.x == m) s_inv[m] = __uint_as_float((uint32_t)(127 - sh) << 23);
+                    for (int c = threadIdx.x; c < cpr; c += GEMV_THREADS) {
+                        uint4 v = *(uint4 *)(xs + m * XS + c * 8);
+                        uint32_t ws[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float lo = __uint_as_float(ws[q] << 16) * sc, hi = __uint_as_float(ws[q] & 0xFFFF0000u) * sc;
-                        ws[q] = as_u32(__floats2half2_rn(lo, hi));
+                        for (int q = 0; q < 4; ++q) {
+                            const float lo = __uint_as_float(ws[q] << 16) * sc, hi = __uint_as_float(ws[q] & 0xFFFF0000u) * sc;
+                            ws[q] = as_u32(__floats2half2_rn(lo, hi));
+                        }
+                        *(uint4 *)(xs + m * XS + c * 8) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
                     }
-                    *(uint4 *)(xs + m * XS + c * 8) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
                 }
             } else {
                 int8_t *xs = reinterpret_cast<int8_t *>(smem);
                 const int cpr = slice_k / 16;
-                for (int idx = threadIdx.x; idx < RT * cpr; idx += GEMV_THREADS) {
-                    const int m = idx / cpr, c = idx % cpr;
-                    uint4 v = make_uint4(0, 0, 0, 0);
-                    // the carrier has a pitch that is a multiple of 128 and is zero beyond K
-                    if (m < M) v = *(const uint4 *)(xq + (int64_t)m * x8_pitch + k_base + c * 16);
-                    *(uint4 *)(xs + m * XS + c * 16) = v;
-                }
+                for (int m = 0; m < RT; ++m)
+                    for (int c = threadIdx.x; c < cpr; c += GEMV_THREADS) {
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        // the carrier has a pitch that is a multiple of 128 and is zero beyond K
+                        if (m < M) v = *(const uint4 *)(xq + (int64_t)m * x8_pitch + k_base + c * 16);
+                        *(uint4 *)(xs + m * XS + c * 16) = v;
+                    }
                 if (threadIdx.x < 16) s_inv[threadIdx.x] = threadIdx.x < M ? dxs[threadIdx.x] * (1.0f / 127.0f) : 0.0f;
             }
             __syncthreads();
+            if (MODE == 0 && threadIdx.x < 16) s_max[threadIdx.x] = 0;  // next slice's maxima start from zero
 
             // ---- stream the tiles of this slice
             float acc[NT][4];
@@ -396,15 +407,18 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
             for (int tb = 0; tb < NT; ++tb)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) acc[tb][i] = 0.0f;
-            const uint8_t *xlane = smem + (size_t)(g * XS + 4 * t) * ES;
-            for (int kb = ks; kb < ke; kb += NBUF) {
+            const uint8_t *xcur = smem + (size_t)(g * XS + 4 * t) * ES;  // this lane's B-fragment base, current tile
+            int to_load = (ke - ks) - NBUF;                              // tiles not yet requested
+            for (int left = ke - ks; left > 0; left -= NBUF) {
                 static_for<NBUF>([&](auto ic) {
                     constexpr int i = decltype(ic)::value;
-                    if (kb + i < ke) {
-                        compute_tile<B, G, NT, MODE>(buf[i], xlane + (size_t)(kb + i - ks) * TILE * ES, XS, ctab, g, t, acc);
-                        if (kb + i + NBUF < ke) {
-                            const size_t off = (size_t)(kb + i + NBUF - ks) * d.tile_bytes;
-                            load_tile<B, GPT>(buf[i], rbp0 + off, prm0 + off, lane);
+                    if (i < left) {
+                        compute_tile<B, G, NT, MODE>(buf[i], xcur, XS, ctab, g, t, acc);
+                        xcur += TILE * ES;
+                        if (to_load > 0) {
+                            load_tile<B, GPT>(buf[i], wl, pl, lane);
+                            wl += d.tile_bytes; pl += d.tile_bytes;
+                            --to_load;
                         }
                     }
                 });
@@ -438,19 +452,29 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                 }
             }
         if (!whole) {
-            // the last CTA to arrive at this row block adds the slots in slot order
-            __threadfence();
+            // the last CTA to arrive at this row block adds the slots in slot order.  The barrier orders
+            // the CTA's partial stores before thread 0's release; its acquire plus the second barrier
+            // make the other CTAs' partials visible to every thread of the last one.
             __syncthreads();
-            if (threadIdx.x == 0) s_last = (atomicAdd(&counters[nb], 1) == n_contrib - 1);
+            if (threadIdx.x == 0) {
+                int old;
+                asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(counters + nb) : "memory");
+                s_last = (old == n_contrib - 1);
+            }
             __syncthreads();
             if (s_last) {
-                __threadfence();
                 const float *pb = partial + (size_t)nb * max_slots * (size_t)(M * TILE);
                 for (int idx = threadIdx.x; idx < M * TILE; idx += GEMV_THREADS) {
                     const int m = idx / TILE, r = idx % TILE;
                     const int64_t n = (int64_t)nb * TILE + r;
                     float sum = 0.0f;
-                    for (int q = 0; q < n_contrib; ++q) sum += __ldcg(pb + (size_t)q * (M * TILE) + idx);
+                    for (int q0 = 0; q0 < n_contrib; q0 += 8) {  // eight independent loads in flight, added in slot order
+                        float v[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) v[i] = (q0 + i < n_contrib) ? __ldcg(pb + (size_t)(q0 + i) * (M * TILE) + idx) : 0.0f;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) sum += v[i];
+                    }
                     if (n < d.N) y[(int64_t)m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(sum));
                 }
                 if (threadIdx.x == 0) counters[nb] = 0;  // leave the workspace ready for the next call
@@ -515,7 +539,7 @@ cudaError_t dispatch_g(const void *layout, const Dims &d, const uint16_t *x, con
 GemvPlan gemv_plan(const Dims &d, int64_t M) {
     GemvPlan p;
     const int64_t T = (int64_t)d.NB * d.KT;
-    int64_t P = (M <= 8 && d.B <= 4 && d.G >= 64) ? 148 * 3 : 148 * 2;
+    int64_t P = (M <= 8 && d.B <= 4 && d.G >= 64) ? 148 * CQ_GEMV_OCC_HI : 148 * 2;
     if (P > T) P = T;
     p.ctas = (int)P;
     int mx = 1;
