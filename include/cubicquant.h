@@ -91,6 +91,11 @@ int cq_unpack(const void *layout, int B, int G, int64_t N, int64_t K, uint8_t *c
 int cq_gemm(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, int64_t M, int64_t N, int64_t K,
             int mode, void *workspace, size_t workspace_bytes, void *stream);
 
+/* Reads back the device status word of a workspace (waits for `stream` first).  CQ_OK, or
+ * CQ_ERR_TIMEOUT when a bounded device-side wait of an earlier cq_gemm on this workspace gave up
+ * (its output is then undefined; re-initialise the workspace before reusing it). */
+int cq_gemm_status(const void *workspace, size_t workspace_bytes, void *stream);
+
 /* Same product with HOST activations and HOST output: copies x_host to the device, runs cq_gemm
  * and copies y back, all on `stream`, then waits for the stream.  x_dev (M*K bf16) and y_dev
  * (M*N bf16) are caller-provided device staging buffers.  Pinned host memory makes the copies

@@ -49,6 +49,8 @@ def lib():
         L.cq_repack.argtypes = [vp, vp, vp, vp, i, i, i64, i64, vp, vp]
         L.cq_unpack.argtypes = [vp, i, i, i64, i64, vp, vp, vp, vp, vp]
         L.cq_gemm.argtypes = [vp, i, i, vp, vp, i64, i64, i64, i, vp, sz, vp]
+        L.cq_gemm_status.argtypes = [vp, sz, vp]
+        L.cq_gemm_status.restype = i
         L.cq_gemm_host.argtypes = [vp, i, i, vp, vp, vp, vp, i64, i64, i64, i, vp, sz, vp]
         L.cq_quantize_a8.argtypes = [vp, i64, i64, vp, vp, vp]
         L.cq_decode_levels.argtypes = [vp, i, i, i64, i64, vp, vp]
@@ -155,6 +157,11 @@ def cq_gemm(pw: PackedWeights, x: torch.Tensor, mode: int = CQ_MODEL_DTYPE, work
     _check(lib().cq_gemm(_ptr(pw.layout), pw.B, pw.G, _ptr(x), _ptr(y), M, pw.N, pw.K, mode, _ptr(workspace),
                          workspace.numel(), _stream()), "cq_gemm")
     return y
+
+
+def cq_gemm_status(workspace: torch.Tensor) -> int:
+    """0, or the negative CQ_ERR_TIMEOUT when a bounded device wait gave up (synchronises the stream)."""
+    return lib().cq_gemm_status(_ptr(workspace), workspace.numel(), _stream())
 
 
 def cq_gemm_host(pw: PackedWeights, x_host: torch.Tensor, y_host: torch.Tensor, x_dev: torch.Tensor,

@@ -20,8 +20,8 @@ Workspace plan_workspace(const Dims &d, int64_t M, int mode) {
     const int64_t Mc = M < 16 ? M : 16;  // rows handled by one small-M launch
     const GemvPlan gp = gemv_plan(d, Mc);
     size_t off = 0;
+    w.status_off = off; off += 256;  // first, so cq_gemm_status finds it without knowing the problem
     w.counters_off = off; w.counters_bytes = align_up((size_t)d.NB * 4, 256); off += w.counters_bytes;
-    w.status_off = off; off += 256;
     w.partial_off = off; w.partial_bytes = align_up((size_t)d.NB * gp.max_slots * Mc * TILE * 4, 256); off += w.partial_bytes;
     if (mode == CQ_DYN_A8) {
         w.x8_off = off; w.x8_bytes = align_up((size_t)(M + 127) / 128 * 128 * Kp, 256); off += w.x8_bytes;
@@ -145,7 +145,7 @@ int cq_gemm(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, in
     cudaStream_t s = (cudaStream_t)stream;
     uint8_t *ws = (uint8_t *)workspace;
     if (M <= 16) return wrap(launch_gemv(layout, d, x, y, M, mode, ws, plan, s));
-    if (gemm_tc_available()) return wrap(launch_gemm_tc(layout, d, x, y, M, mode, ws, plan, s));
+    if (mode == CQ_MODEL_DTYPE && gemm_tc_available()) return wrap(launch_gemm_tc(layout, d, x, y, M, mode, ws, plan, s));
     // conservative route: 16 rows at a time through the small-M kernel (weights re-streamed per chunk)
     for (int64_t m0 = 0; m0 < M; m0 += 16) {
         const int64_t mc = (M - m0 < 16) ? (M - m0) : 16;
@@ -153,6 +153,17 @@ int cq_gemm(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, in
         if (e != cudaSuccess) return wrap(e);
     }
     return CQ_OK;
+}
+
+int cq_gemm_status(const void *workspace, size_t workspace_bytes, void *stream) {
+    if (!workspace || workspace_bytes < 512) return CQ_ERR_INVALID_ARG;
+    // the status word is the first word of every workspace (plan_workspace)
+    int host = 0;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return wrap(e);
+    e = cudaMemcpy(&host, (const uint8_t *)workspace, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return wrap(e);
+    return host == 0 ? CQ_OK : CQ_ERR_TIMEOUT;
 }
 
 int cq_gemm_host(const void *layout, int B, int G, const uint16_t *x_host, uint16_t *y_host, uint16_t *x_dev,

@@ -1,14 +1,476 @@
-// Large-M tcgen05 / TMEM GEMM (placeholder translation unit until the kernel lands).
+// Large-M packed GEMM on the 5th-generation tensor cores (Section 5.3 dense path, re-done for
+// sm_100a): weights stay packed in HBM and are decoded into bf16 shared-memory operand tiles
+// right before tcgen05.mma consumes them; accumulators live in TMEM.
+//
+// Roles inside a CTA (one 128-row x BN-token output tile):
+//   warp 0      producer: bulk-copies raw layout tiles (codes + co-located group parameters) and
+//               TMA-loads activation tiles x[BN x 64] (128-byte swizzle) into a ring of stages
+//   warp 1      allocates TMEM, issues tcgen05.mma (one elected lane), commits to mbarriers
+//   warps 2..5  decode: raw tile -> s_g * q(|k|/M) * sign in fp32 (Eq. cubic, Horner form of
+//               Eq. gpu-horner on the power-of-two-normalised code), rounded to bf16 and stored in
+//               the K-major 128-byte-swizzled layout the MMA reads; then the epilogue
+//               (tcgen05.ld -> bf16 -> y)
+// Weights sit on the MMA's M side (TMEM lane = output channel), tokens on its N side, so any
+// token count maps to a legal instruction shape and each epilogue thread owns one output channel.
+//
+// Every wait on an mbarrier is bounded: a wait that runs out sets a status word in global memory
+// and makes the role leave its loop; the CTA still releases TMEM and exits.
+#include <cuda.h>
+
+#include <utility>
+
 #include "cq_common.cuh"
 #include "cq_internal.h"
 
 namespace cq {
 
-int gemm_tc_available() { return 0; }
+int gemm_tc_available() { return 1; }
 
-cudaError_t launch_gemm_tc(const void *, const Dims &, const uint16_t *, uint16_t *, int64_t, int, uint8_t *,
-                           const Workspace &, cudaStream_t) {
-    return cudaErrorNotSupported;
+namespace {
+
+constexpr int TC_THREADS = 192;
+constexpr int A_STAGE_BYTES = 128 * 128;  // 128 rows x 64 bf16
+constexpr int RAW_STAGES = 2;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;  // about two seconds
+
+template <int... I, class F>
+__device__ __forceinline__ void static_for_impl(F &&f, std::integer_sequence<int, I...>) {
+    (f(std::integral_constant<int, I>{}), ...);
+}
+template <int N, class F>
+__device__ __forceinline__ void static_for(F &&f) {
+    static_for_impl(static_cast<F &&>(f), std::make_integer_sequence<int, N>{});
+}
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred P1;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, P1;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false (and a status word) when the barrier did not flip within the limit.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *status, int code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            atomicCAS(status, 0, code);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_2d(void *smem, const CUtensorMap *map, uint64_t *bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(smem)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void bulk_load(void *smem, const void *gmem, uint32_t bytes, uint64_t *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(smem)), "l"(gmem), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc], bf16 inputs, fp32 accumulate
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major operand tile with 128-byte swizzle: rows are 128
+// bytes, eight-row groups 1024 bytes apart, descriptor version 1 (sm_100), layout type 2.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+           ((uint64_t)2 << 61);
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t idesc_bf16(int BN) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+// ---------------------------------------------------------------- decode helpers
+template <int B, int P>
+__device__ __forceinline__ uint32_t pair_codes_smem(const uint32_t (&w)[2 * B]) {
+    uint32_t u2 = 0;
+    static_for<plane_count(B)>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        constexpr int pw = plane_width(B, i), ppw = 16 / pw;
+        constexpr int W = plane_word_base(B, i) + P / ppw, pos = (P % ppw) * pw;
+        constexpr uint32_t m = ((1u << pw) - 1u) * 0x00010001u;
+        u2 |= ((w[W] >> pos) & m) << plane_bit_offset(B, i);
+    });
+    return u2;
+}
+
+struct RowScaled { float as, bs, cs, s; bool fix; };  // s * (a rho, b rho^2, c rho^3); flag: reserved pattern present
+
+template <int B>
+__device__ __forceinline__ RowScaled scaled_coef(uint2 p) {
+    RowScaled c;
+    c.s = __uint_as_float(p.x & 0x7FFFFFFFu);
+    c.fix = (p.x >> 31) != 0;
+    if constexpr (B >= 3) {
+        constexpr float rho = (float)(1 << (B - 1)) / (float)((1 << (B - 1)) - 1);
+        constexpr float rho2 = rho * rho, rho3 = rho * rho * rho;
+        const __half2 ab = *reinterpret_cast<const __half2 *>(&p.y);
+        const float a = __low2float(ab), b = __high2float(ab), cc = (1.0f - a) - b;
+        c.as = c.s * (a * rho);
+        c.bs = c.s * (b * rho2);
+        c.cs = c.s * (cc * rho3);
+    } else {
+        c.as = c.bs = c.cs = 0.0f;
+    }
+    return c;
+}
+
+// Reconstructed weight s * sign(k) * q(|k| / M) of stored code u, fp32.
+template <int B>
+__device__ __forceinline__ float weight_of_code(unsigned u, const RowScaled &c) {
+    if constexpr (B == 1) {
+        return u ? c.s : -c.s;
+    } else if constexpr (B == 2) {
+        return u == 0 ? 0.0f : c.s * (float)((int)u - 2);
+    } else {
+        // T = (u - 2^(B-1)) / 2^(B-1) exactly: integer into the mantissa of 2^23, one FMA
+        constexpr float inv = 1.0f / (float)(1 << (B - 1));
+        float T = fmaf(__uint_as_float(u | 0x4B000000u), inv, -(8388608.0f + (float)(1 << (B - 1))) * inv);
+        if (c.fix && u == 0) T = 0.0f;
+        const float at = fabsf(T);
+        return T * fmaf(at, fmaf(at, c.cs, c.bs), c.as);
+    }
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&v);
+}
+
+struct TcParams {
+    const uint8_t *layout;
+    uint16_t *y;
+    int *status;
+    Dims d;
+    int M;
+    int raw_stage_bytes;  // tile_bytes rounded up to 1024
+};
+
+// ---------------------------------------------------------------- the kernel (model dtype)
+template <int B, int G, int BN>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
+    constexpr int GPT = TILE / G;
+    constexpr int STAGES = BN == 256 ? 3 : 4;          // ring of 64-wide k blocks
+    constexpr int B_STAGE_BYTES = BN * 128;
+    constexpr uint32_t TMEM_COLS = BN < 32 ? 32 : BN;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *sA = smem;                                        // STAGES x 16 KB
+    uint8_t *sB = sA + STAGES * A_STAGE_BYTES;                 // STAGES x BN x 128 B
+    uint8_t *sRaw = sB + STAGES * B_STAGE_BYTES;               // RAW_STAGES x raw_stage_bytes
+    uint64_t *bars = reinterpret_cast<uint64_t *>(sRaw + RAW_STAGES * prm.raw_stage_bytes);
+    uint64_t *a_full = bars, *b_full = bars + STAGES, *st_empty = bars + 2 * STAGES;
+    uint64_t *raw_full = bars + 3 * STAGES, *raw_empty = raw_full + RAW_STAGES, *acc_full = raw_empty + RAW_STAGES;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+
+    const Dims &d = prm.d;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nb = blockIdx.x, mt = blockIdx.y;
+    const int KT = d.KT;            // layout tiles along K
+    const int NKB = 2 * KT;         // 64-wide k blocks
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&a_full[s], 4); mbar_init(&b_full[s], 1); mbar_init(&st_empty[s], 1); }
+        for (int s = 0; s < RAW_STAGES; ++s) { mbar_init(&raw_full[s], 1); mbar_init(&raw_empty[s], 4); }
+        mbar_init(acc_full, 1);
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ===== producer
+        if (lane == 0) {
+            const uint8_t *tiles = prm.layout + (size_t)nb * KT * (size_t)d.tile_bytes;
+            bool ok = true;
+            for (int kb = 0; kb < NKB && ok; ++kb) {
+                if ((kb & 1) == 0) {
+                    const int t = kb >> 1, rs = t % RAW_STAGES;
+                    if (t >= RAW_STAGES) ok = mbar_wait(&raw_empty[rs], ((t / RAW_STAGES) - 1) & 1, prm.status, 1);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(&raw_full[rs], (uint32_t)d.tile_bytes);
+                    bulk_load(sRaw + rs * prm.raw_stage_bytes, tiles + (size_t)t * d.tile_bytes, (uint32_t)d.tile_bytes, &raw_full[rs]);
+                }
+                const int s = kb % STAGES;
+                if (kb >= STAGES) ok = mbar_wait(&st_empty[s], ((kb / STAGES) - 1) & 1, prm.status, 2);
+                if (!ok) break;
+                mbar_arrive_expect_tx(&b_full[s], B_STAGE_BYTES);
+                tma_load_2d(sB + s * B_STAGE_BYTES, &xmap, &b_full[s], kb * 64, mt * BN);
+            }
+        }
+    } else if (warp == 1) {
+        // ===== MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16(BN);
+            bool ok = true;
+            for (int kb = 0; kb < NKB && ok; ++kb) {
+                const int s = kb % STAGES;
+                const uint32_t ph = (kb / STAGES) & 1;
+                ok = mbar_wait(&a_full[s], ph, prm.status, 3) && mbar_wait(&b_full[s], ph, prm.status, 4);
+                if (!ok) break;
+                tc_fence_after();
+                const uint64_t adesc = smem_desc_sw128(smem_u32(sA + s * A_STAGE_BYTES));
+                const uint64_t bdesc = smem_desc_sw128(smem_u32(sB + s * B_STAGE_BYTES));
+#pragma unroll
+                for (int k = 0; k < 4; ++k)  // four K = 16 steps, 32 bytes apart inside the swizzle atom
+                    umma_bf16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                umma_commit(&st_empty[s]);  // frees the stage when these MMAs have read it
+            }
+            umma_commit(acc_full);
+        }
+    } else {
+        // ===== decoders (warps 2..5), then epilogue
+        const int dw = warp - 2, g = lane >> 2, t = lane & 3;
+        bool ok = true;
+        for (int tile = 0; tile < KT && ok; ++tile) {
+            const int rs = tile % RAW_STAGES;
+            ok = mbar_wait(&raw_full[rs], (tile / RAW_STAGES) & 1, prm.status, 5);
+            if (!ok) break;
+            const uint8_t *raw = sRaw + rs * prm.raw_stage_bytes;
+#pragma unroll 1
+            for (int half_k = 0; half_k < 2 && ok; ++half_k) {
+                const int kb = 2 * tile + half_k, s = kb % STAGES;
+                if (kb >= STAGES) ok = mbar_wait(&st_empty[s], ((kb / STAGES) - 1) & 1, prm.status, 6);
+                if (!ok) break;
+                uint8_t *a_stage = sA + s * A_STAGE_BYTES;
+#pragma unroll 1
+                for (int rbi = 0; rbi < 2; ++rbi) {
+                    const int rb = 2 * dw + rbi;
+                    const uint8_t *rbp = raw + rb * 256 * B;
+                    uint32_t w[2 * B];
+                    {
+                        constexpr int NFQ = (2 * B) / 4;
+#pragma unroll
+                        for (int q = 0; q < NFQ; ++q) {
+                            const uint4 v = *(const uint4 *)(rbp + (q * 32 + lane) * 16);
+                            w[4 * q + 0] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+                        }
+                        if constexpr ((2 * B) % 4 != 0) {
+                            const uint2 v = *(const uint2 *)(rbp + NFQ * 512 + lane * 8);
+                            w[4 * NFQ + 0] = v.x; w[4 * NFQ + 1] = v.y;
+                        }
+                    }
+                    const uint8_t *prow = raw + d.code_bytes + ((rb * 16 + g) * GPT) * 8;
+                    // rows g (low) and g + 8 (high) of this row block: byte offsets of their smem rows
+                    uint8_t *row_lo = a_stage + (rb * 2 + 0) * 1024 + g * 128;
+                    uint8_t *row_hi = a_stage + (rb * 2 + 1) * 1024 + g * 128;
+                    auto do_half = [&](auto hk) {
+                        constexpr int HK = decltype(hk)::value;
+                        constexpr int NGH = G >= 64 ? 1 : 64 / G;       // groups inside one 64-wide k block
+                        constexpr int CPG = 4 / NGH;                    // 16-wide chunks per such group
+                        static_for<NGH>([&](auto gg) {
+                            constexpr int gh = decltype(gg)::value;
+                            constexpr int gi = (64 * HK + 16 * CPG * gh) / G;
+                            const RowScaled c_lo = scaled_coef<B>(*(const uint2 *)(prow + gi * 8));
+                            const RowScaled c_hi = scaled_coef<B>(*(const uint2 *)(prow + (8 * GPT + gi) * 8));
+                            static_for<CPG>([&](auto jj) {
+                                constexpr int jl = CPG * gh + decltype(jj)::value, j = 4 * HK + jl;  // 16-wide chunk
+                                const uint32_t u0 = pair_codes_smem<B, 4 * j + 0>(w), u1 = pair_codes_smem<B, 4 * j + 1>(w);
+                                const uint32_t u2 = pair_codes_smem<B, 4 * j + 2>(w), u3 = pair_codes_smem<B, 4 * j + 3>(w);
+                                uint2 lo, hi;  // four consecutive k of one row = 8 bytes
+                                lo.x = pack_bf16(weight_of_code<B>(u0 & 0xFFFFu, c_lo), weight_of_code<B>(u0 >> 16, c_lo));
+                                lo.y = pack_bf16(weight_of_code<B>(u2 & 0xFFFFu, c_lo), weight_of_code<B>(u2 >> 16, c_lo));
+                                hi.x = pack_bf16(weight_of_code<B>(u1 & 0xFFFFu, c_hi), weight_of_code<B>(u1 >> 16, c_hi));
+                                hi.y = pack_bf16(weight_of_code<B>(u3 & 0xFFFFu, c_hi), weight_of_code<B>(u3 >> 16, c_hi));
+                                // k offset inside the 64-wide block: 16 jl + 4 t -> 16-byte chunk 2 jl + t/2, swizzled by the row
+                                const int chunk = (2 * jl + (t >> 1)) ^ g;
+                                const int off = chunk * 16 + (t & 1) * 8;
+                                *(uint2 *)(row_lo + off) = lo;
+                                *(uint2 *)(row_hi + off) = hi;
+                            });
+                        });
+                    };
+                    if (half_k == 0) do_half(std::integral_constant<int, 0>{});
+                    else do_half(std::integral_constant<int, 1>{});
+                }
+                fence_proxy_async();   // generic-proxy stores -> visible to the tensor core's async proxy
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&a_full[s]);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&raw_empty[rs]);
+        }
+        // ----- epilogue: TMEM lane = output channel, column = token
+        if (ok) ok = mbar_wait(acc_full, 0, prm.status, 7);
+        tc_fence_after();
+        if (ok) {
+            const int q4 = warp & 3;                       // TMEM lane quarter this warp may access
+            const int64_t n = (int64_t)nb * TILE + q4 * 32 + lane;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)c0, r);
+                tmem_ld_wait();
+                if (n < d.N) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int64_t m = (int64_t)mt * BN + c0 + i;
+                        if (m < prm.M) prm.y[m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(r[i])));
+                    }
+                }
+            }
+        }
+    }
+    if (*reinterpret_cast<volatile int *>(prm.status) != 0) {
+        // a wait gave up: give copies that are still in flight time to land before shared memory is released
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+template <int B, int G, int BN>
+cudaError_t launch_bn(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int *status,
+                      cudaStream_t st) {
+    EncodeTiledFn enc = encode_tiled();
+    if (!enc) return cudaErrorNotSupported;
+    CUtensorMap xmap;
+    const cuuint64_t dims[2] = {(cuuint64_t)d.K, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)d.K * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)BN};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t *>(x), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+    constexpr int STAGES = BN == 256 ? 3 : 4;
+    TcParams p;
+    p.layout = (const uint8_t *)layout; p.y = y; p.status = status; p.d = d; p.M = (int)M;
+    p.raw_stage_bytes = (d.tile_bytes + 1023) / 1024 * 1024;
+    const size_t smem = 1024 + (size_t)STAGES * (A_STAGE_BYTES + BN * 128) + (size_t)RAW_STAGES * p.raw_stage_bytes + 256;
+    auto kern = gemm_tc_kernel<B, G, BN>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    dim3 grid((unsigned)d.NB, (unsigned)((M + BN - 1) / BN));
+    kern<<<grid, TC_THREADS, smem, st>>>(xmap, p);
+    return cudaGetLastError();
+}
+
+template <int B, int G>
+cudaError_t launch_g(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int *status,
+                     cudaStream_t st) {
+    if (M <= 32) return launch_bn<B, G, 32>(layout, d, x, y, M, status, st);
+    if (M <= 64) return launch_bn<B, G, 64>(layout, d, x, y, M, status, st);
+    if (M <= 128 || (M <= 512 && d.NB * ((M + 127) / 128) <= 148)) return launch_bn<B, G, 128>(layout, d, x, y, M, status, st);
+    return launch_bn<B, G, 256>(layout, d, x, y, M, status, st);
+}
+
+template <int B>
+cudaError_t launch_b(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int *status,
+                     cudaStream_t st) {
+    switch (d.G) {
+        case 32: return launch_g<B, 32>(layout, d, x, y, M, status, st);
+        case 64: return launch_g<B, 64>(layout, d, x, y, M, status, st);
+        default: return launch_g<B, 128>(layout, d, x, y, M, status, st);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
+                           uint8_t *ws, const Workspace &plan, cudaStream_t st) {
+    if (mode != 0) return cudaErrorNotSupported;
+    int *status = reinterpret_cast<int *>(ws + plan.status_off);
+    switch (d.B) {
+        case 1: return launch_b<1>(layout, d, x, y, M, status, st);
+        case 2: return launch_b<2>(layout, d, x, y, M, status, st);
+        case 3: return launch_b<3>(layout, d, x, y, M, status, st);
+        case 4: return launch_b<4>(layout, d, x, y, M, status, st);
+        case 5: return launch_b<5>(layout, d, x, y, M, status, st);
+        case 6: return launch_b<6>(layout, d, x, y, M, status, st);
+        case 7: return launch_b<7>(layout, d, x, y, M, status, st);
+        default: return launch_b<8>(layout, d, x, y, M, status, st);
+    }
 }
 
 }  // namespace cq

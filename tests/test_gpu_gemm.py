@@ -95,3 +95,30 @@ def test_repeatable_bitwise_and_workspace_reuse():
     y1 = cq.cq_gemm(c.pw, x, 0, ws).clone()
     y2 = cq.cq_gemm(c.pw, x, 0, ws).clone()
     assert torch.equal(y1.view(torch.int16), y2.view(torch.int16))  # fixed split-K order: deterministic
+
+
+@pytest.mark.parametrize("G", [32, 64, 128])
+@pytest.mark.parametrize("B", ALL_B)
+def test_tensor_core_gemm_all_widths_and_groups(B, G):
+    # M = 40 runs the tcgen05 path with a 64-token tile; ragged N and K, reserved codes, a zero group
+    N, K = 200, 352 if G == 32 else 384
+    c = logical_case(N, K, B, G, seed=160 + B)
+    if B > 1:
+        c.k[5, 3:40] = -(1 << (B - 1))
+    c.s[17, 1] = 0.0
+    c = Case(c.k, c.s, c.a, c.b, B, G)
+    x = datagen.activations(40, K, seed=161)
+    y, ref = run_both(c, x, cq.CQ_MODEL_DTYPE)
+    check_y(y, ref, f"tc B={B} G={G}")
+
+
+@pytest.mark.parametrize("M", [513, 700])
+def test_tensor_core_gemm_wide_token_tile(M):
+    # more than 512 rows: 256-token tiles, last tile ragged
+    c = encoded_case("normal", 384, 1024, 4, 128, seed=170, sigma=0.015)
+    x = datagen.activations(M, 1024, seed=171)
+    y, ref = run_both(c, x, cq.CQ_MODEL_DTYPE)
+    check_y(y, ref, f"tc M={M}")
+    ws = torch.zeros(cq.cq_workspace_bytes(4, 128, M, 384, 1024, 0), dtype=torch.uint8, device="cuda")
+    cq.cq_gemm(c.pw, x_to_device(x), 0, ws)
+    assert cq.cq_gemm_status(ws) == 0
