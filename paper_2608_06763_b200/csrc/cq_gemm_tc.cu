@@ -6,8 +6,8 @@
 //   warp 0      producer: bulk-copies raw layout tiles (codes + co-located group parameters) and
 //               TMA-loads activation tiles x[BN x 64] (128-byte swizzle) into a ring of stages
 //   warp 1      allocates TMEM, issues tcgen05.mma (one elected lane), commits to mbarriers
-//   warps 2..5  decode: raw tile -> s_g * q(|k|/M) * sign in fp32 (Eq. cubic, Horner form of
-//               Eq. gpu-horner on the power-of-two-normalised code), rounded to bf16 and stored in
+//   warps 2..17 decode: raw tile -> s_g * q(|k|/M) * sign (Eq. cubic; q by the half2 Horner form of
+//               Eq. gpu-horner on the power-of-two-normalised code, scale in fp32), rounded to bf16 and stored in
 //               the K-major 128-byte-swizzled layout the MMA reads; then the epilogue
 //               (tcgen05.ld -> bf16 -> y)
 // Weights sit on the MMA's M side (TMEM lane = output channel), tokens on its N side, so any
@@ -17,9 +17,8 @@
 // and makes the role leave its loop; the CTA still releases TMEM and exits.
 #include <cuda.h>
 
-#include <utility>
-
 #include "cq_common.cuh"
+#include "cq_decode.cuh"
 #include "cq_internal.h"
 
 namespace cq {
@@ -28,19 +27,11 @@ int gemm_tc_available() { return 1; }
 
 namespace {
 
-constexpr int TC_THREADS = 192;
+constexpr int DEC_WARPS = 16;                 // decoder / epilogue warps
+constexpr int TC_THREADS = 64 + 32 * DEC_WARPS;
 constexpr int A_STAGE_BYTES = 128 * 128;  // 128 rows x 64 bf16
 constexpr int RAW_STAGES = 2;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;  // about two seconds
-
-template <int... I, class F>
-__device__ __forceinline__ void static_for_impl(F &&f, std::integer_sequence<int, I...>) {
-    (f(std::integral_constant<int, I>{}), ...);
-}
-template <int N, class F>
-__device__ __forceinline__ void static_for(F &&f) {
-    static_for_impl(static_cast<F &&>(f), std::make_integer_sequence<int, N>{});
-}
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -141,59 +132,15 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int BN) {
 }
 
 // ---------------------------------------------------------------- decode helpers
-template <int B, int P>
-__device__ __forceinline__ uint32_t pair_codes_smem(const uint32_t (&w)[2 * B]) {
-    uint32_t u2 = 0;
-    static_for<plane_count(B)>([&](auto ic) {
-        constexpr int i = decltype(ic)::value;
-        constexpr int pw = plane_width(B, i), ppw = 16 / pw;
-        constexpr int W = plane_word_base(B, i) + P / ppw, pos = (P % ppw) * pw;
-        constexpr uint32_t m = ((1u << pw) - 1u) * 0x00010001u;
-        u2 |= ((w[W] >> pos) & m) << plane_bit_offset(B, i);
-    });
-    return u2;
-}
-
-struct RowScaled { float as, bs, cs, s; bool fix; };  // s * (a rho, b rho^2, c rho^3); flag: reserved pattern present
-
-template <int B>
-__device__ __forceinline__ RowScaled scaled_coef(uint2 p) {
-    RowScaled c;
-    c.s = __uint_as_float(p.x & 0x7FFFFFFFu);
-    c.fix = (p.x >> 31) != 0;
-    if constexpr (B >= 3) {
-        constexpr float rho = (float)(1 << (B - 1)) / (float)((1 << (B - 1)) - 1);
-        constexpr float rho2 = rho * rho, rho3 = rho * rho * rho;
-        const __half2 ab = *reinterpret_cast<const __half2 *>(&p.y);
-        const float a = __low2float(ab), b = __high2float(ab), cc = (1.0f - a) - b;
-        c.as = c.s * (a * rho);
-        c.bs = c.s * (b * rho2);
-        c.cs = c.s * (cc * rho3);
-    } else {
-        c.as = c.bs = c.cs = 0.0f;
-    }
-    return c;
-}
-
-// Reconstructed weight s * sign(k) * q(|k| / M) of stored code u, fp32.
-template <int B>
-__device__ __forceinline__ float weight_of_code(unsigned u, const RowScaled &c) {
-    if constexpr (B == 1) {
-        return u ? c.s : -c.s;
-    } else if constexpr (B == 2) {
-        return u == 0 ? 0.0f : c.s * (float)((int)u - 2);
-    } else {
-        // T = (u - 2^(B-1)) / 2^(B-1) exactly: integer into the mantissa of 2^23, one FMA
-        constexpr float inv = 1.0f / (float)(1 << (B - 1));
-        float T = fmaf(__uint_as_float(u | 0x4B000000u), inv, -(8388608.0f + (float)(1 << (B - 1))) * inv);
-        if (c.fix && u == 0) T = 0.0f;
-        const float at = fabsf(T);
-        return T * fmaf(at, fmaf(at, c.cs, c.bs), c.as);
-    }
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+// Two reconstructed weights s * sign(k) * q(|k| / M) of one pair, rounded to bf16 (the dense path
+// of Section 5.3 rounds the temporary operand to the activation dtype).  q is evaluated in half2
+// (11-bit significand, finer than the bf16 it is rounded to), the scale is applied in fp32.
+template <int B, int P, bool FIX>
+__device__ __forceinline__ uint32_t weight_pair_bf16(const uint32_t (&w)[2 * B], const RowCoef &c) {
+    const __half2 T = pair_T<B, P>(w);
+    const uint32_t q = level_pair<B, FIX>(T, c);
+    const float2 f = __half22float2(as_h2(q));
+    const __nv_bfloat162 v = __floats2bfloat162_rn(f.x * c.s, f.y * c.s);
     return *reinterpret_cast<const uint32_t *>(&v);
 }
 
@@ -207,15 +154,20 @@ struct TcParams {
 };
 
 // ---------------------------------------------------------------- the kernel (model dtype)
-template <int B, int G, int BN>
+constexpr int tc_stages(int BN, int NACC) { return BN * NACC >= 512 ? 2 : (BN == 256 ? 3 : 4); }
+
+// One CTA computes 128 output channels x (NACC * BN) tokens: NACC accumulators of BN columns share
+// every decoded weight tile, which halves the decode work per flop at NACC = 2.
+template <int B, int G, int BN, int NACC>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
     constexpr int GPT = TILE / G;
-    constexpr int STAGES = BN == 256 ? 3 : 4;          // ring of 64-wide k blocks
-    constexpr int B_STAGE_BYTES = BN * 128;
-    constexpr uint32_t TMEM_COLS = BN < 32 ? 32 : BN;
-    extern __shared__ __align__(1024) uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    constexpr int STAGES = tc_stages(BN, NACC);        // ring of 64-wide k blocks
+    constexpr int B_TILE_BYTES = BN * 128;             // one TMA box: BN tokens x 64 k
+    constexpr int B_STAGE_BYTES = NACC * B_TILE_BYTES;
+    constexpr int BNT = BN * NACC;                     // tokens per CTA
+    constexpr uint32_t TMEM_COLS = BNT < 32 ? 32 : BNT;
+    extern __shared__ __align__(1024) uint8_t smem[];  // 1024-byte alignment is what the swizzled tiles need
     uint8_t *sA = smem;                                        // STAGES x 16 KB
     uint8_t *sB = sA + STAGES * A_STAGE_BYTES;                 // STAGES x BN x 128 B
     uint8_t *sRaw = sB + STAGES * B_STAGE_BYTES;               // RAW_STAGES x raw_stage_bytes
@@ -230,9 +182,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
     const int KT = d.KT;            // layout tiles along K
     const int NKB = 2 * KT;         // 64-wide k blocks
 
+    if ((smem_u32(smem) & 1023u) != 0) {  // cannot happen with the alignment attribute; never run misaligned
+        if (threadIdx.x == 0) atomicCAS(prm.status, 0, 9);
+        return;
+    }
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&a_full[s], 4); mbar_init(&b_full[s], 1); mbar_init(&st_empty[s], 1); }
-        for (int s = 0; s < RAW_STAGES; ++s) { mbar_init(&raw_full[s], 1); mbar_init(&raw_empty[s], 4); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&a_full[s], DEC_WARPS); mbar_init(&b_full[s], 1); mbar_init(&st_empty[s], 1); }
+        for (int s = 0; s < RAW_STAGES; ++s) { mbar_init(&raw_full[s], 1); mbar_init(&raw_empty[s], DEC_WARPS); }
         mbar_init(acc_full, 1);
         fence_barrier_init();
     }
@@ -262,7 +218,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                 if (kb >= STAGES) ok = mbar_wait(&st_empty[s], ((kb / STAGES) - 1) & 1, prm.status, 2);
                 if (!ok) break;
                 mbar_arrive_expect_tx(&b_full[s], B_STAGE_BYTES);
-                tma_load_2d(sB + s * B_STAGE_BYTES, &xmap, &b_full[s], kb * 64, mt * BN);
+#pragma unroll
+                for (int a = 0; a < NACC; ++a)
+                    tma_load_2d(sB + s * B_STAGE_BYTES + a * B_TILE_BYTES, &xmap, &b_full[s], kb * 64, mt * BNT + a * BN);
             }
         }
     } else if (warp == 1) {
@@ -277,78 +235,81 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                 if (!ok) break;
                 tc_fence_after();
                 const uint64_t adesc = smem_desc_sw128(smem_u32(sA + s * A_STAGE_BYTES));
-                const uint64_t bdesc = smem_desc_sw128(smem_u32(sB + s * B_STAGE_BYTES));
 #pragma unroll
-                for (int k = 0; k < 4; ++k)  // four K = 16 steps, 32 bytes apart inside the swizzle atom
-                    umma_bf16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                for (int a = 0; a < NACC; ++a) {
+                    const uint64_t bdesc = smem_desc_sw128(smem_u32(sB + s * B_STAGE_BYTES + a * B_TILE_BYTES));
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)  // four K = 16 steps, 32 bytes apart inside the swizzle atom
+                        umma_bf16(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                }
                 umma_commit(&st_empty[s]);  // frees the stage when these MMAs have read it
             }
             umma_commit(acc_full);
         }
     } else {
-        // ===== decoders (warps 2..5), then epilogue
+        // ===== decoders (warps 2..17), then epilogue.  Per 64-wide k block, decoder dw owns row block
+        // dw / 2 and the two 16-wide chunks 2 (dw % 2), 2 (dw % 2) + 1 of the block.
         const int dw = warp - 2, g = lane >> 2, t = lane & 3;
+        const int rb = dw >> 1, jh = dw & 1;
         bool ok = true;
         for (int tile = 0; tile < KT && ok; ++tile) {
             const int rs = tile % RAW_STAGES;
             ok = mbar_wait(&raw_full[rs], (tile / RAW_STAGES) & 1, prm.status, 5);
             if (!ok) break;
             const uint8_t *raw = sRaw + rs * prm.raw_stage_bytes;
+            const uint8_t *rbp = raw + rb * 256 * B;
+            uint32_t w[2 * B];
+            {
+                constexpr int NFQ = (2 * B) / 4;
+#pragma unroll
+                for (int q = 0; q < NFQ; ++q) {
+                    const uint4 v = *(const uint4 *)(rbp + (q * 32 + lane) * 16);
+                    w[4 * q + 0] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+                }
+                if constexpr ((2 * B) % 4 != 0) {
+                    const uint2 v = *(const uint2 *)(rbp + NFQ * 512 + lane * 8);
+                    w[4 * NFQ + 0] = v.x; w[4 * NFQ + 1] = v.y;
+                }
+            }
+            const uint8_t *prow = raw + d.code_bytes + ((rb * 16 + g) * GPT) * 8;
 #pragma unroll 1
             for (int half_k = 0; half_k < 2 && ok; ++half_k) {
                 const int kb = 2 * tile + half_k, s = kb % STAGES;
                 if (kb >= STAGES) ok = mbar_wait(&st_empty[s], ((kb / STAGES) - 1) & 1, prm.status, 6);
                 if (!ok) break;
                 uint8_t *a_stage = sA + s * A_STAGE_BYTES;
-#pragma unroll 1
-                for (int rbi = 0; rbi < 2; ++rbi) {
-                    const int rb = 2 * dw + rbi;
-                    const uint8_t *rbp = raw + rb * 256 * B;
-                    uint32_t w[2 * B];
-                    {
-                        constexpr int NFQ = (2 * B) / 4;
-#pragma unroll
-                        for (int q = 0; q < NFQ; ++q) {
-                            const uint4 v = *(const uint4 *)(rbp + (q * 32 + lane) * 16);
-                            w[4 * q + 0] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
-                        }
-                        if constexpr ((2 * B) % 4 != 0) {
-                            const uint2 v = *(const uint2 *)(rbp + NFQ * 512 + lane * 8);
-                            w[4 * NFQ + 0] = v.x; w[4 * NFQ + 1] = v.y;
-                        }
-                    }
-                    const uint8_t *prow = raw + d.code_bytes + ((rb * 16 + g) * GPT) * 8;
-                    // rows g (low) and g + 8 (high) of this row block: byte offsets of their smem rows
-                    uint8_t *row_lo = a_stage + (rb * 2 + 0) * 1024 + g * 128;
-                    uint8_t *row_hi = a_stage + (rb * 2 + 1) * 1024 + g * 128;
-                    auto do_half = [&](auto hk) {
-                        constexpr int HK = decltype(hk)::value;
-                        constexpr int NGH = G >= 64 ? 1 : 64 / G;       // groups inside one 64-wide k block
-                        constexpr int CPG = 4 / NGH;                    // 16-wide chunks per such group
-                        static_for<NGH>([&](auto gg) {
-                            constexpr int gh = decltype(gg)::value;
-                            constexpr int gi = (64 * HK + 16 * CPG * gh) / G;
-                            const RowScaled c_lo = scaled_coef<B>(*(const uint2 *)(prow + gi * 8));
-                            const RowScaled c_hi = scaled_coef<B>(*(const uint2 *)(prow + (8 * GPT + gi) * 8));
-                            static_for<CPG>([&](auto jj) {
-                                constexpr int jl = CPG * gh + decltype(jj)::value, j = 4 * HK + jl;  // 16-wide chunk
-                                const uint32_t u0 = pair_codes_smem<B, 4 * j + 0>(w), u1 = pair_codes_smem<B, 4 * j + 1>(w);
-                                const uint32_t u2 = pair_codes_smem<B, 4 * j + 2>(w), u3 = pair_codes_smem<B, 4 * j + 3>(w);
-                                uint2 lo, hi;  // four consecutive k of one row = 8 bytes
-                                lo.x = pack_bf16(weight_of_code<B>(u0 & 0xFFFFu, c_lo), weight_of_code<B>(u0 >> 16, c_lo));
-                                lo.y = pack_bf16(weight_of_code<B>(u2 & 0xFFFFu, c_lo), weight_of_code<B>(u2 >> 16, c_lo));
-                                hi.x = pack_bf16(weight_of_code<B>(u1 & 0xFFFFu, c_hi), weight_of_code<B>(u1 >> 16, c_hi));
-                                hi.y = pack_bf16(weight_of_code<B>(u3 & 0xFFFFu, c_hi), weight_of_code<B>(u3 >> 16, c_hi));
-                                // k offset inside the 64-wide block: 16 jl + 4 t -> 16-byte chunk 2 jl + t/2, swizzled by the row
-                                const int chunk = (2 * jl + (t >> 1)) ^ g;
-                                const int off = chunk * 16 + (t & 1) * 8;
-                                *(uint2 *)(row_lo + off) = lo;
-                                *(uint2 *)(row_hi + off) = hi;
-                            });
+                // rows g (low) and g + 8 (high) of the row block: their 128-byte rows in the stage
+                uint8_t *row_lo = a_stage + (rb * 2 + 0) * 1024 + g * 128;
+                uint8_t *row_hi = a_stage + (rb * 2 + 1) * 1024 + g * 128;
+                auto do_unit = [&](auto jq) {
+                    constexpr int JQ = decltype(jq)::value;        // pair of chunks 2 JQ, 2 JQ + 1 of the tile
+                    constexpr int gi = (32 * JQ) / G;              // both chunks lie in this group
+                    const uint2 p_lo = *(const uint2 *)(prow + gi * 8), p_hi = *(const uint2 *)(prow + (8 * GPT + gi) * 8);
+                    const RowCoef c_lo = make_coef<B>(p_lo), c_hi = make_coef<B>(p_hi);
+                    const bool fix = B > 1 && __any_sync(0xffffffffu, (p_lo.x | p_hi.x) >> 31);  // reserved pattern present
+                    auto emit = [&](auto fx) {
+                        constexpr bool FIX = decltype(fx)::value;
+                        static_for<2>([&](auto jc) {
+                            constexpr int j = 2 * JQ + decltype(jc)::value, jl = j & 3;
+                            uint2 lo, hi;  // four consecutive k of one row = 8 bytes
+                            lo.x = weight_pair_bf16<B, 4 * j + 0, FIX>(w, c_lo);
+                            hi.x = weight_pair_bf16<B, 4 * j + 1, FIX>(w, c_hi);
+                            lo.y = weight_pair_bf16<B, 4 * j + 2, FIX>(w, c_lo);
+                            hi.y = weight_pair_bf16<B, 4 * j + 3, FIX>(w, c_hi);
+                            // k offset inside the 64-wide block: 16 jl + 4 t -> 16-byte chunk 2 jl + t/2, swizzled by the row
+                            const int chunk = (2 * jl + (t >> 1)) ^ g;
+                            const int off = chunk * 16 + (t & 1) * 8;
+                            *(uint2 *)(row_lo + off) = lo;
+                            *(uint2 *)(row_hi + off) = hi;
                         });
                     };
-                    if (half_k == 0) do_half(std::integral_constant<int, 0>{});
-                    else do_half(std::integral_constant<int, 1>{});
+                    if (!fix) emit(std::false_type{}); else emit(std::true_type{});
+                };
+                switch (half_k * 2 + jh) {
+                    case 0: do_unit(std::integral_constant<int, 0>{}); break;
+                    case 1: do_unit(std::integral_constant<int, 1>{}); break;
+                    case 2: do_unit(std::integral_constant<int, 2>{}); break;
+                    default: do_unit(std::integral_constant<int, 3>{}); break;
                 }
                 fence_proxy_async();   // generic-proxy stores -> visible to the tensor core's async proxy
                 __syncwarp();
@@ -362,16 +323,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
         tc_fence_after();
         if (ok) {
             const int q4 = warp & 3;                       // TMEM lane quarter this warp may access
+            const int cp = dw >> 2;                        // which of four column parts
             const int64_t n = (int64_t)nb * TILE + q4 * 32 + lane;
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            for (int c0 = cp * 32; c0 < BNT; c0 += 128) {
                 uint32_t r[32];
                 tmem_ld32(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)c0, r);
                 tmem_ld_wait();
                 if (n < d.N) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        const int64_t m = (int64_t)mt * BN + c0 + i;
+                        const int64_t m = (int64_t)mt * BNT + c0 + i;
                         if (m < prm.M) prm.y[m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(r[i])));
                     }
                 }
@@ -405,7 +367,7 @@ EncodeTiledFn encode_tiled() {
     return fn;
 }
 
-template <int B, int G, int BN>
+template <int B, int G, int BN, int NACC>
 cudaError_t launch_bn(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int *status,
                       cudaStream_t st) {
     EncodeTiledFn enc = encode_tiled();
@@ -419,19 +381,19 @@ cudaError_t launch_bn(const void *layout, const Dims &d, const uint16_t *x, uint
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
-    constexpr int STAGES = BN == 256 ? 3 : 4;
+    constexpr int STAGES = tc_stages(BN, NACC);
     TcParams p;
     p.layout = (const uint8_t *)layout; p.y = y; p.status = status; p.d = d; p.M = (int)M;
     p.raw_stage_bytes = (d.tile_bytes + 1023) / 1024 * 1024;
-    const size_t smem = 1024 + (size_t)STAGES * (A_STAGE_BYTES + BN * 128) + (size_t)RAW_STAGES * p.raw_stage_bytes + 256;
-    auto kern = gemm_tc_kernel<B, G, BN>;
+    const size_t smem = (size_t)STAGES * (A_STAGE_BYTES + NACC * BN * 128) + (size_t)RAW_STAGES * p.raw_stage_bytes + 256;
+    auto kern = gemm_tc_kernel<B, G, BN, NACC>;
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    dim3 grid((unsigned)d.NB, (unsigned)((M + BN - 1) / BN));
+    dim3 grid((unsigned)d.NB, (unsigned)((M + BN * NACC - 1) / (BN * NACC)));
     kern<<<grid, TC_THREADS, smem, st>>>(xmap, p);
     return cudaGetLastError();
 }
@@ -439,10 +401,11 @@ cudaError_t launch_bn(const void *layout, const Dims &d, const uint16_t *x, uint
 template <int B, int G>
 cudaError_t launch_g(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int *status,
                      cudaStream_t st) {
-    if (M <= 32) return launch_bn<B, G, 32>(layout, d, x, y, M, status, st);
-    if (M <= 64) return launch_bn<B, G, 64>(layout, d, x, y, M, status, st);
-    if (M <= 128 || (M <= 512 && d.NB * ((M + 127) / 128) <= 148)) return launch_bn<B, G, 128>(layout, d, x, y, M, status, st);
-    return launch_bn<B, G, 256>(layout, d, x, y, M, status, st);
+    if (M <= 32) return launch_bn<B, G, 32, 1>(layout, d, x, y, M, status, st);
+    if (M <= 64) return launch_bn<B, G, 64, 1>(layout, d, x, y, M, status, st);
+    if (M <= 128) return launch_bn<B, G, 128, 1>(layout, d, x, y, M, status, st);
+    if (M <= 256) return launch_bn<B, G, 256, 1>(layout, d, x, y, M, status, st);
+    return launch_bn<B, G, 256, 2>(layout, d, x, y, M, status, st);
 }
 
 template <int B>

@@ -17,9 +17,8 @@
 //
 // Dynamic A8 uses the INT8 m16n8k32 MMA on signed carriers looked up in a per-warp table of the
 // group's non-negative carriers (Eq. carrier), int32 group partials, fp32 rescale (Eq. a8-output).
-#include <utility>
-
 #include "cq_common.cuh"
+#include "cq_decode.cuh"
 #include "cq_internal.h"
 
 namespace cq {
@@ -32,15 +31,6 @@ constexpr int MAX_SUB = 16;    // K tiles staged at a time (bounds shared memory
 #ifndef CQ_GEMV_OCC_HI
 #define CQ_GEMV_OCC_HI 3       // resident CTAs per SM asked of the compiler for the light variants
 #endif
-
-template <int... I, class F>
-__device__ __forceinline__ void static_for_impl(F &&f, std::integer_sequence<int, I...>) {
-    (f(std::integral_constant<int, I>{}), ...);
-}
-template <int N, class F>
-__device__ __forceinline__ void static_for(F &&f) {
-    static_for_impl(static_cast<F &&>(f), std::make_integer_sequence<int, N>{});
-}
 
 __device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm(
@@ -66,15 +56,6 @@ __device__ __forceinline__ uint2 ld_stream8(const void *p) {
     return v;
 }
 
-// fp16 bit patterns built with integer arithmetic only (so they are compile-time constants)
-constexpr uint32_t h2dup(uint32_t h) { return h | (h << 16); }
-constexpr uint32_t half_pow2(int e) { return (uint32_t)((e + 15) << 10); }                      // 2^e, -14 <= e <= 15
-constexpr uint32_t half_neg_pow2_plus(int q, int c) {                                            // -(2^q + c), c < 2^q, q <= 10
-    return 0x8000u | (uint32_t)((q + 15) << 10) | (uint32_t)(c << (10 - q));
-}
-__device__ __forceinline__ __half2 as_h2(uint32_t v) { return *reinterpret_cast<__half2 *>(&v); }
-__device__ __forceinline__ uint32_t as_u32(__half2 v) { return *reinterpret_cast<uint32_t *>(&v); }
-
 template <int B, int GPT>
 struct TileRegs {
     uint32_t w[2 * B];
@@ -98,81 +79,6 @@ __device__ __forceinline__ void load_tile(TileRegs<B, GPT> &r, const uint8_t *wl
     for (int gi = 0; gi < GPT; ++gi) {
         r.prm[0][gi] = ld_stream8(pl + gi * 8);
         r.prm[1][gi] = ld_stream8(pl + (8 * GPT + gi) * 8);
-    }
-}
-
-// Two stored codes of pair P as packed 16-bit integers (u_lo | u_hi << 16).
-template <int B, int P>
-__device__ __forceinline__ uint32_t pair_codes(const uint32_t (&w)[2 * B]) {
-    uint32_t u2 = 0;
-    static_for<plane_count(B)>([&](auto ic) {
-        constexpr int i = decltype(ic)::value;
-        constexpr int pw = plane_width(B, i), ppw = 16 / pw;
-        constexpr int W = plane_word_base(B, i) + P / ppw, pos = (P % ppw) * pw;
-        constexpr uint32_t m = ((1u << pw) - 1u) * 0x00010001u;
-        u2 |= ((w[W] >> pos) & m) << plane_bit_offset(B, i);
-    });
-    return u2;
-}
-
-// Pair P as half2 of the normalised signed code:  B >= 3: T = k / 2^(B-1);  B <= 2: k itself.
-// The stored code lands in the fp16 mantissa under exponent bits 0x6400 (value 1024 + u 2^pos);
-// one exact FMA removes the offset and the position scale.
-template <int B, int P>
-__device__ __forceinline__ __half2 pair_T(const uint32_t (&w)[2 * B]) {
-    if constexpr (plane_count(B) == 1) {
-        constexpr int PPW = 16 / B, W = P / PPW, pos0 = (P % PPW) * B;
-        // B = 1 keeps the field off mantissa bit 0 (the offset constant must stay representable);
-        // other widths shift by 8 when the field would leave the 10 mantissa bits
-        constexpr int shl = (B == 1 && pos0 <= 6) ? 1 : 0;
-        constexpr int shr = (B == 1) ? (pos0 <= 6 ? 0 : 6) : (pos0 + B > 10 ? 8 : 0);
-        constexpr int pos = pos0 + shl - shr;
-        const uint32_t word = shl ? (w[W] << shl) : (shr ? (w[W] >> shr) : w[W]);
-        constexpr uint32_t m = (((1u << B) - 1u) << pos) * 0x00010001u;
-        const uint32_t hbits = (word & m) | 0x64006400u;
-        constexpr uint32_t sc = (B == 1) ? half_pow2(1 - pos) : (B == 2) ? half_pow2(-pos) : half_pow2(-(pos + B - 1));
-        constexpr uint32_t off = (B == 1) ? half_neg_pow2_plus(11 - pos, 1)
-                               : (B == 2) ? half_neg_pow2_plus(10 - pos, 2)
-                                          : half_neg_pow2_plus(10 - pos - (B - 1), 1);
-        return __hfma2(as_h2(hbits), as_h2(h2dup(sc)), as_h2(h2dup(off)));
-    } else {
-        const uint32_t hbits = pair_codes<B, P>(w) | 0x64006400u;
-        constexpr uint32_t sc = half_pow2(-(B - 1)), off = half_neg_pow2_plus(10 - (B - 1), 1);
-        return __hfma2(as_h2(hbits), as_h2(h2dup(sc)), as_h2(h2dup(off)));
-    }
-}
-
-struct RowCoef { __half2 a2, b2, c2; float s; };
-
-// Coefficients of q as a polynomial in T = k / 2^(B-1):  t = |T| rho, rho = 2^(B-1) / M, so
-// q = |T| (a rho + |T| (b rho^2 + |T| c rho^3)).
-template <int B>
-__device__ __forceinline__ RowCoef make_coef(uint2 p) {
-    RowCoef c;
-    c.s = __uint_as_float(p.x & 0x7FFFFFFFu);
-    if constexpr (B >= 3) {
-        constexpr float rho = (float)(1 << (B - 1)) / (float)((1 << (B - 1)) - 1);
-        constexpr float rho2 = rho * rho, rho3 = rho * rho * rho;
-        const __half2 ab = as_h2(p.y);
-        const float a = __low2float(ab), b = __high2float(ab), cc = (1.0f - a) - b;
-        c.a2 = __float2half2_rn(a * rho);
-        c.b2 = __float2half2_rn(b * rho2);
-        c.c2 = __float2half2_rn(cc * rho3);
-    }
-    return c;
-}
-
-template <int B, bool FIX>
-__device__ __forceinline__ uint32_t level_pair(__half2 T, const RowCoef &c) {
-    if constexpr (FIX) {  // reserved pattern: T = -1 (B >= 3) or k = -2 (B = 2) decodes to zero
-        const __half2 bad = __float2half2_rn(B == 2 ? -2.0f : -1.0f);
-        T = __hmul2(T, __hne2(T, bad));
-    }
-    if constexpr (B >= 3) {
-        const __half2 at = __habs2(T);
-        return as_u32(__hmul2(T, __hfma2(at, __hfma2(at, c.c2, c.b2), c.a2)));
-    } else {
-        return as_u32(T);
     }
 }
 
