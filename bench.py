@@ -33,6 +33,9 @@ SWEEP_B = [1, 2, 3, 4, 6, 8]
 SWEEP_G = [32, 64, 128]
 SWEEP_N = SWEEP_K = 8192
 L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the W4 G128 8192x8192 M=1 GEMV, from the
+# ncu capture summarised in profiles/gemv_w4g128_8192_m1.md (algorithmic bytes: 37.78 MB)
+NCU_TRAFFIC_W4G128_BYTES = 37816320
 
 
 def eff_bytes(N, K, B, G):
@@ -106,6 +109,93 @@ def build_case(cq, torch, N, K, B, G, seed, copies):
     pws = [pw] + [cq.PackedWeights(pw.layout.clone(), B, G, N, K) for _ in range(copies - 1)]
     del dk, codes
     return pws
+
+
+
+def make_packed_cuda(cq, datagen, N, K, B, G, seed):
+    k, s, a, b = datagen.logical_quantized_cuda(N, K, B, G, seed)
+    codes = cq.cq_pack_codes(k, B)
+    pw = cq.cq_repack(codes, s, a, b, B, G, N, K)
+    del k, codes
+    return pw
+
+
+def time_graph(torch, stream, fn, reps):
+    """ms per call of fn() captured `reps` times in one CUDA graph (best of 3 replays)."""
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        for i in range(reps):
+            fn(i)
+    g.replay(); stream.synchronize()
+    best = 1e30
+    for _ in range(3):
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream); g.replay(); a1.record(stream); stream.synchronize()
+        best = min(best, a0.elapsed_time(a1) / reps)
+    return best
+
+
+def extra_suites(torch, cq, datagen, stream, peaks):
+    """Secondary workloads reported beside the headline: prefill-scale GEMM (Llama-3-70B MLP shapes,
+    M = 4096, W3/W4 G128), Llama-3-8B decode linears at M in {1,4,8,16}, and the model-dtype versus
+    Dynamic-A8 crossover in M."""
+    out = {}
+    # ---- prefill GEMM
+    gemm = []
+    M = 4096
+    for name, K, N in datagen.LLAMA70B_MLP_SHAPES:
+        x = datagen.activations_cuda(M, K, seed=4)
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        for B in (3, 4):
+            pw = make_packed_cuda(cq, datagen, N, K, B, 128, 4)
+            ws = torch.zeros(cq.cq_workspace_bytes(B, 128, M, N, K, 0), dtype=torch.uint8, device="cuda")
+            for _ in range(2):
+                cq.cq_gemm(pw, x, cq.CQ_MODEL_DTYPE, ws, y)
+            ms = time_graph(torch, stream, lambda i: cq.cq_gemm(pw, x, cq.CQ_MODEL_DTYPE, ws, y), 3)
+            tf = 2.0 * M * N * K / (ms * 1e-3) / 1e12
+            gemm.append({"shape": name, "K": K, "N": N, "M": M, "B": B, "G": 128, "mode": "model_dtype",
+                         "ms": round(ms, 4), "tflops": round(tf, 1),
+                         "frac_of_measured_bf16_burst": round(tf / peaks["bf16_tflops"], 4)})
+            del pw, ws
+        del x, y
+        torch.cuda.empty_cache()
+    out["gemm_prefill"] = gemm
+    # ---- decode linears and crossover
+    dec, cross = [], []
+    for name, K, N in datagen.LLAMA8B_SHAPES:
+        pws = {B: make_packed_cuda(cq, datagen, N, K, B, 128, 2) for B in (4, 8)}
+        copies = {B: [pws[B]] + [cq.PackedWeights(pws[B].layout.clone(), B, 128, N, K)
+                                 for _ in range(int(np.ceil(2 * L2_BYTES / pws[B].layout.numel())))] for B in (4, 8)}
+        for M in (1, 4, 8, 16, 64, 256, 1024):
+            x = datagen.activations_cuda(M, K, seed=3, outlier_cols=0.01)
+            y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+            for B in (4, 8):
+                t = {}
+                for mode in (cq.CQ_MODEL_DTYPE, cq.CQ_DYN_A8):
+                    if mode == cq.CQ_DYN_A8 and M not in (1, 16, 64, 256, 1024):
+                        continue
+                    ws = torch.zeros(cq.cq_workspace_bytes(B, 128, M, N, K, mode), dtype=torch.uint8, device="cuda")
+                    cp = copies[B]
+                    fn = lambda i: cq.cq_gemm(cp[i % len(cp)], x, mode, ws, y)
+                    fn(0)
+                    t[mode] = time_graph(torch, stream, fn, max(len(cp), 8) if M <= 64 else 4)
+                if B == 4 and M <= 16:
+                    dec.append({"shape": name, "K": K, "N": N, "M": M, "us": round(t[0] * 1e3, 2),
+                                "gbs": round(eff_bytes(N, K, 4, 128) / (t[0] * 1e-3) / 1e9, 1)})
+                if 1 in t:
+                    cross.append({"shape": name, "B": B, "M": M, "us_model": round(t[0] * 1e3, 2),
+                                  "us_a8": round(t[1] * 1e3, 2), "model_over_a8": round(t[0] / t[1], 3)})
+        del pws, copies
+        torch.cuda.empty_cache()
+    out["decode_linears_w4g128"] = dec
+    out["crossover"] = cross
+    first = {}
+    for c in cross:
+        key = f"{c['shape']}-W{c['B']}"
+        if c["model_over_a8"] > 1.0 and key not in first:
+            first[key] = c["M"]
+    out["crossover_first_M_where_a8_is_faster"] = first
+    return out
 
 
 def run_ours(args, rank, world):
@@ -199,7 +289,7 @@ def run_ours(args, rank, world):
         achieved = dom_bytes / (dom["us"] * 1e-6) / 1e9
         roofline = {"bound": "hbm", "kernel": "gemv_kernel<B=4,G=128,NT=1,model>", "achieved": round(achieved, 1),
                     "peak": peaks["hbm_gbs"], "peak_source": peaks["source"] + " (burst copy)", "unit": "GB/s",
-                    "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": None,
+                    "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": NCU_TRAFFIC_W4G128_BYTES,
                     "bytes_per_launch": dom_bytes, "us_per_launch": dom["us"]}
 
         # end to end through the host-buffer entry point: pinned host x in, y out, every call
@@ -226,6 +316,14 @@ def run_ours(args, rank, world):
                "h2d_bytes_per_step": len(cases) * M * K * 2, "d2h_bytes_per_step": len(cases) * M * N * 2,
                "ms_per_step": round(e2e_ms, 4)}
 
+        extras = {}
+        if args.suite == "all" and world == 1:
+            for c in cases:
+                c["pws"] = None
+            cases.clear()
+            torch.cuda.empty_cache()
+            extras = extra_suites(torch, cq, datagen, stream, peaks)
+
     out = None
     if rank == 0:
         cpu = cpu_baseline_sample() if world == 1 else None
@@ -238,6 +336,7 @@ def run_ours(args, rank, world):
                           "timing": "one CUDA graph of all timed steps, CUDA events around its replay"},
                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": n_launch,
                "clocks": clocks.summary(), "cases": per_case}
+        out.update(extras)
     if world > 1:
         dist.destroy_process_group()
     return out
@@ -298,6 +397,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--suite", default="all", choices=["sweep", "all"],
+                    help="sweep: headline GEMV sweep only; all: also prefill GEMM, decode linears, crossover")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", 0))

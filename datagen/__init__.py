@@ -159,3 +159,45 @@ def logical_quantized(N: int, K: int, B: int, G: int, seed: int, name: str = "Q"
 LLAMA8B_SHAPES = [("qkv", 4096, 6144), ("o", 4096, 4096),
                   ("gate_up", 4096, 28672), ("down", 14336, 4096)]
 LLAMA70B_MLP_SHAPES = [("gate_up", 8192, 57344), ("down", 28672, 8192)]
+
+
+def logical_quantized_cuda(N: int, K: int, B: int, G: int, seed: int, device="cuda"):
+    """Same recipe as ``logical_quantized`` (bell-shaped signed codes, shape parameters in the
+    strictly monotone domain, scales in [0.03, 0.09]) drawn with torch's seeded generator on the
+    GPU, for tensors too large to draw with numpy in reasonable time.  Returns torch tensors
+    (k int8 [N, K], s fp32, a fp16, b fp16 of shape [N, K/G]) on ``device``.  The stream differs
+    from the numpy one; consumers that need the values on the CPU copy them back."""
+    import torch
+    assert K % G == 0
+    gen = torch.Generator(device=device)
+    gen.manual_seed(int(seed) * 1000003 + B * 131 + G)
+    k = torch.empty((N, K), dtype=torch.int8, device=device)
+    rows = max(1, (1 << 26) // K)  # draw in slabs to bound temporary memory
+    for r0 in range(0, N, rows):
+        r1 = min(N, r0 + rows)
+        u = torch.rand((r1 - r0, K), generator=gen, device=device, dtype=torch.float32)
+        if B == 1:
+            k[r0:r1] = torch.where(u < 0.5, -1, 1).to(torch.int8)
+        else:
+            Mx = (1 << (B - 1)) - 1
+            d = (u - 0.5).clamp(-0.4999999, 0.4999999)
+            v = -(0.22 * Mx + 0.35) * torch.sign(d) * torch.log1p(-2.0 * d.abs())
+            k[r0:r1] = v.round().clamp(-Mx, Mx).to(torch.int8)
+    n = N * (K // G)
+    s = (0.03 + 0.06 * torch.rand(n, generator=gen, device=device)).to(torch.float32).reshape(N, K // G)
+    a = (0.5 + 0.5 * torch.rand(n, generator=gen, device=device)).to(torch.float16).reshape(N, K // G)
+    b = (-0.3 * torch.rand(n, generator=gen, device=device)).to(torch.float16).reshape(N, K // G)
+    return k, s, a, b
+
+
+def activations_cuda(M: int, K: int, seed: int, outlier_cols: float = 0.0, outlier_scale: float = 20.0, device="cuda"):
+    """bf16 N(0,1) activations [M, K] drawn on the GPU (optionally a seeded set of columns scaled)."""
+    import torch
+    gen = torch.Generator(device=device)
+    gen.manual_seed(int(seed) * 7919 + 17)
+    x = torch.randn((M, K), generator=gen, device=device, dtype=torch.float32)
+    n_out = int(outlier_cols * K)
+    if n_out > 0:
+        cols = torch.randperm(K, generator=gen, device=device)[:n_out]
+        x[:, cols] *= outlier_scale
+    return x.to(torch.bfloat16)
