@@ -104,6 +104,32 @@ int cq_gemm_host(const void *layout, int B, int G, const uint16_t *x_host, uint1
                  uint16_t *y_dev, int64_t M, int64_t N, int64_t K, int mode, void *workspace, size_t workspace_bytes,
                  void *stream);
 
+/* Small-M product (M <= 16, model dtype) for callers that cannot hand the library any scratch
+ * memory.  (The paper has no counterpart to this call; it exists for integration reasons only.)
+ *
+ * Who needs it: code that runs where device allocation is off limits, for example an operator
+ * plug-in on the request path of an inference server.  Such a plug-in is given its input and output
+ * tensors and nothing else; it may not call cudaMalloc (it synchronises the whole device and can
+ * fail under the server's fixed memory budget) and has no hook into the host framework's allocator
+ * to ask for a workspace.  For those callers the split-K scratch (arrival counters and partial
+ * sums) comes from an array of CQ_STATIC_SCRATCH_BYTES that is compiled into the library and
+ * occupies that much memory on every GPU that loads it, until the process exits.
+ *
+ *   - Same arguments and result as cq_gemm(..., CQ_MODEL_DTYPE, ...) without the workspace; all
+ *     pointers are device pointers owned by the caller, 16-byte aligned; enqueues on `stream`.
+ *   - No allocation of any kind is made, neither by this call nor by anything it calls.
+ *   - CQ_ERR_WORKSPACE when the problem needs more scratch than the built-in array holds
+ *     (cq_workspace_bytes(B, G, M, N, K, CQ_MODEL_DTYPE) > CQ_STATIC_SCRATCH_BYTES);
+ *     CQ_ERR_UNSUPPORTED for M > 16 or an unsupported format.
+ *   - The first call on each device looks up the array's device address (with that device current).
+ *     Make that first call during start-up, before any stream capture begins.
+ *   - Every call on a device shares the one array and finds in it what the previous call left; the
+ *     call clears the counters it relies on before launching.  Two calls whose kernels may overlap
+ *     on the GPU (different streams, or host threads) race on the array: serialise them. */
+#define CQ_STATIC_SCRATCH_BYTES (8u << 20)
+int cq_gemv_static(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, int64_t M, int64_t N, int64_t K,
+                   void *stream);
+
 /* Pieces of the path exposed for parity tests. */
 
 /* Dynamic-A8 activation quantiser (Eq. a8-activation-scale, Eq. a8-activation-quantization):

@@ -51,6 +51,8 @@ def lib():
         L.cq_gemm.argtypes = [vp, i, i, vp, vp, i64, i64, i64, i, vp, sz, vp]
         L.cq_gemm_status.argtypes = [vp, sz, vp]
         L.cq_gemm_status.restype = i
+        L.cq_gemv_static.argtypes = [vp, i, i, vp, vp, i64, i64, i64, vp]
+        L.cq_gemv_static.restype = i
         L.cq_gemm_host.argtypes = [vp, i, i, vp, vp, vp, vp, i64, i64, i64, i, vp, sz, vp]
         L.cq_quantize_a8.argtypes = [vp, i64, i64, vp, vp, vp]
         L.cq_decode_levels.argtypes = [vp, i, i, i64, i64, vp, vp]
@@ -162,6 +164,17 @@ def cq_gemm(pw: PackedWeights, x: torch.Tensor, mode: int = CQ_MODEL_DTYPE, work
 def cq_gemm_status(workspace: torch.Tensor) -> int:
     """0, or the negative CQ_ERR_TIMEOUT when a bounded device wait gave up (synchronises the stream)."""
     return lib().cq_gemm_status(_ptr(workspace), workspace.numel(), _stream())
+
+
+def cq_gemv_static(pw: PackedWeights, x: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    """Small-M product (M <= 16, model dtype) that takes its scratch from the array built into the
+    library: for callers that may not allocate.  Calls on one device must not overlap."""
+    assert x.dtype == torch.bfloat16 and x.dim() == 2 and x.shape[1] == pw.K
+    M = x.shape[0]
+    y = out if out is not None else torch.empty((M, pw.N), dtype=torch.bfloat16, device=x.device)
+    _check(lib().cq_gemv_static(_ptr(pw.layout), pw.B, pw.G, _ptr(x), _ptr(y), M, pw.N, pw.K, _stream()),
+           "cq_gemv_static")
+    return y
 
 
 def cq_gemm_host(pw: PackedWeights, x_host: torch.Tensor, y_host: torch.Tensor, x_dev: torch.Tensor,
