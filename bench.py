@@ -98,6 +98,22 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def max_over_ranks(value, world, device="cuda"):
+    """The slowest rank's time (or any scalar): all-reduce MAX over the process group."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(step_bytes, ms_per_step, world):
+    """Whole-job GB/s of `world` replicas that each process step_bytes per step (weak scaling)."""
+    return world * step_bytes / (ms_per_step * 1e-3) / 1e9
+
+
 # ----------------------------------------------------------------------------- our arm
 def build_case(cq, torch, N, K, B, G, seed, copies):
     import datagen
@@ -256,13 +272,10 @@ def run_ours(args, rank, world):
                 graph.replay()
             stream.synchronize()
         torch.cuda.synchronize()
-        if world > 1:
-            t = torch.tensor([t_ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            t_ms = float(t.item())
+        t_ms = max_over_ranks(t_ms, world)
         ms_per_step = t_ms / args.steps
         step_bytes = sum(c["bytes"] for c in cases)
-        value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+        value = aggregate_throughput(step_bytes, ms_per_step, world)
 
         # per-case and dominant-kernel timing: a graph of launches of one case over its rotating copies
         def time_case(c, reps=None):
@@ -308,11 +321,8 @@ def run_ours(args, rank, world):
                 cq.cq_gemm_host(c["pws"][(i + 2) % len(c["pws"])], xh, yh, x, y, cq.CQ_MODEL_DTYPE, ws)
         torch.cuda.synchronize()
         e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
-        if world > 1:
-            t = torch.tensor([e2e_ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e = {"value": round(world * step_bytes / (e2e_ms * 1e-3) / 1e9, 2), "unit": "GB/s",
+        e2e_ms = max_over_ranks(e2e_ms, world)
+        e2e = {"value": round(aggregate_throughput(step_bytes, e2e_ms, world), 2), "unit": "GB/s",
                "h2d_bytes_per_step": len(cases) * M * K * 2, "d2h_bytes_per_step": len(cases) * M * N * 2,
                "ms_per_step": round(e2e_ms, 4)}
 
