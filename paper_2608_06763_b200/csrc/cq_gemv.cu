@@ -17,6 +17,8 @@
 //
 // Dynamic A8 uses the INT8 m16n8k32 MMA on signed carriers looked up in a per-warp table of the
 // group's non-negative carriers (Eq. carrier), int32 group partials, fp32 rescale (Eq. a8-output).
+#include <cstdlib>
+
 #include "cq_common.cuh"
 #include "cq_decode.cuh"
 #include "cq_internal.h"
@@ -222,6 +224,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
     int8_t *ctab = nullptr;
     if constexpr (MODE == 1 && B >= 3) ctab = reinterpret_cast<int8_t *>(smem) + RT * (MAX_SUB * TILE + XS_PAD) + warp * 16 * L;
 
+    bool first_slice = true;
     for (int64_t tile = t_begin; tile < t_end;) {
         const int nb = (int)(tile / d.KT), kb_begin = (int)(tile % d.KT);
         const int kb_end = (int)min((int64_t)d.KT, kb_begin + (t_end - tile));
@@ -239,7 +242,40 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
             const uint8_t *wl = tile0 + warp * 256 * B + lane * 16;                     // next tile to load (codes)
             const uint8_t *pl = tile0 + d.code_bytes + ((warp * 16 + g) * GPT) * 8;      // next tile to load (params)
 
-            // first weight loads go out before the activations are touched
+            // The activations, the workspace and y may be produced or still used by the kernel launched
+            // before this one: wait for it (a no-op unless the launch allowed programmatic overlap), then
+            // let the next kernel's CTAs start as soon as there is room for them.
+            if (first_slice) {
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+                first_slice = false;
+            }
+            __syncthreads();  // previous slice fully consumed
+
+            // ---- request the activation slice first (asynchronous copies straight into shared memory),
+            // so that it does not queue behind the burst of weight loads issued next.  Thread c owns the
+            // 16-byte chunk c of every token row (a slice has at most 256 chunks per row).
+            const int cpr = MODE == 0 ? slice_k / 8 : slice_k / 16;
+            const int c = threadIdx.x;
+            if (c < cpr) {
+                for (int m = 0; m < RT; ++m) {
+                    uint8_t *dst = smem + ((size_t)m * XS) * ES + (size_t)c * 16;
+                    const void *src = nullptr;
+                    if (m < M) {
+                        if constexpr (MODE == 0) {
+                            const int64_t k = k_base + (int64_t)c * 8;
+                            if (k < d.K) src = x + (int64_t)m * d.K + k;   // K % 8 == 0 always
+                        } else {
+                            src = xq + (int64_t)m * x8_pitch + k_base + c * 16;  // pitch multiple of 128, zero beyond K
+                        }
+                    }
+                    if (src) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+                    else *(uint4 *)dst = make_uint4(0, 0, 0, 0);
+                }
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+
+            // ---- first weight loads
             TileRegs<B, GPT> buf[NBUF];
             static_for<NBUF>([&](auto ic) {
                 constexpr int i = decltype(ic)::value;
@@ -249,31 +285,24 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                 }
             });
 
-            // ---- stage the activation slice [k_base, k_base + slice_k) for RT token rows
-            __syncthreads();  // previous slice fully consumed
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
             if constexpr (MODE == 0) {
                 __half *xs = reinterpret_cast<__half *>(smem);
-                const int cpr = slice_k / 8;  // 16-byte chunks per row
-                // pass 1: raw bf16 into shared memory, row maxima of |x| (as bf16 bit patterns) into s_max
-                for (int m = 0; m < RT; ++m) {
+                // pass 1: row maxima of |x| (as bf16 bit patterns) from the chunks this thread copied
+                for (int m = 0; m < M; ++m) {
                     unsigned mx = 0;
-                    for (int c = threadIdx.x; c < cpr; c += GEMV_THREADS) {
-                        const int64_t k = k_base + (int64_t)c * 8;
-                        uint4 v = make_uint4(0, 0, 0, 0);
-                        if (m < M && k < d.K) v = *(const uint4 *)(x + (int64_t)m * d.K + k);  // K % 8 == 0 always
-                        *(uint4 *)(xs + m * XS + c * 8) = v;
+                    if (c < cpr) {
+                        const uint4 v = *(const uint4 *)(xs + m * XS + c * 8);
                         const uint32_t ws[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                         for (int q = 0; q < 4; ++q) { mx = max(mx, ws[q] & 0x7FFFu); mx = max(mx, (ws[q] >> 16) & 0x7FFFu); }
                     }
-                    if (m < M) {
-                        mx = __reduce_max_sync(0xffffffffu, mx);
-                        if (lane == 0 && mx) atomicMax(&s_max[m], mx);
-                    }
+                    mx = __reduce_max_sync(0xffffffffu, mx);
+                    if (lane == 0 && mx) atomicMax(&s_max[m], mx);
                 }
                 __syncthreads();
                 // pass 2: every thread derives the power-of-two scale that puts the row maximum in
-                // [2^14, 2^15) and converts the chunks it wrote
+                // [2^14, 2^15) and converts the chunks it owns
                 for (int m = 0; m < M; ++m) {
                     const unsigned mb = s_max[m];
                     const int ef = (int)((mb >> 7) & 0xFF);          // biased exponent of the maximum
@@ -281,7 +310,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                     sh = max(min(sh, 100), -100);
                     const float sc = __uint_as_float((uint32_t)(127 + sh) << 23);   // 2^sh
                     if (threadIdx.x == m) s_inv[m] = __uint_as_float((uint32_t)(127 - sh) << 23);
-                    for (int c = threadIdx.x; c < cpr; c += GEMV_THREADS) {
+                    if (c < cpr) {
                         uint4 v = *(uint4 *)(xs + m * XS + c * 8);
                         uint32_t ws[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -293,15 +322,6 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                     }
                 }
             } else {
-                int8_t *xs = reinterpret_cast<int8_t *>(smem);
-                const int cpr = slice_k / 16;
-                for (int m = 0; m < RT; ++m)
-                    for (int c = threadIdx.x; c < cpr; c += GEMV_THREADS) {
-                        uint4 v = make_uint4(0, 0, 0, 0);
-                        // the carrier has a pitch that is a multiple of 128 and is zero beyond K
-                        if (m < M) v = *(const uint4 *)(xq + (int64_t)m * x8_pitch + k_base + c * 16);
-                        *(uint4 *)(xs + m * XS + c * 16) = v;
-                    }
                 if (threadIdx.x < 16) s_inv[threadIdx.x] = threadIdx.x < M ? dxs[threadIdx.x] * (1.0f / 127.0f) : 0.0f;
             }
             __syncthreads();
@@ -410,8 +430,20 @@ cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, con
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    kern<<<P, GEMV_THREADS, smem, st>>>((const uint8_t *)layout, d, x, xq, x8_pitch, dxs, y, M, max_slots, partial, counters);
-    return cudaGetLastError();
+    // Programmatic dependent launch: this kernel may begin (and prefetch weights) while the previous
+    // kernel of the stream drains; it waits for that kernel before touching anything but the weights.
+    static const bool use_pdl = getenv("CQ_NO_PDL") == nullptr;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)P);
+    cfg.blockDim = dim3(GEMV_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = use_pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, (const uint8_t *)layout, d, x, xq, x8_pitch, dxs, y, M, max_slots, partial, counters);
 }
 
 template <int B, int G>
