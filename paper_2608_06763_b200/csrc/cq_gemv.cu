@@ -198,14 +198,21 @@ __device__ __forceinline__ void compute_tile(const TileRegs<B, TILE / G> &r, con
 }
 
 // CTA index that owns linear tile `tile` when T tiles are cut into P runs [floor(c T / P), floor((c+1) T / P)).
-__host__ __device__ inline int owner_of(int64_t tile, int64_t T, int64_t P) { return (int)(((tile + 1) * P - 1) / T); }
+// Runs are cut on a "virtual" line in which every row block is KT tiles preceded by E overhead
+// units: a CTA whose run crosses into a new row block pays a second prologue and a second combine,
+// worth about E tiles, so it is given that many tiles fewer.  V = NB (KT + E) units are cut into P
+// runs [floor(c V / P), floor((c+1) V / P)); owner_of gives the CTA that holds tile (nb, kb).
+__host__ __device__ inline int owner_of(int nb, int kb, int KT, int E, int64_t V, int64_t P) {
+    const int64_t v = (int64_t)nb * (KT + E) + E + kb;
+    return (int)(((v + 1) * P - 1) / V);
+}
 
 // ------------------------------------------------------------------------------------------
 // MODE 0: model dtype.  MODE 1: Dynamic A8 (xq = int8 carrier [M][x8_pitch], dxs = row scales).
 template <int B, int G, int NT, int MODE>
 __global__ void __launch_bounds__(GEMV_THREADS, (NT == 1 && B <= 4 && G >= 64) ? CQ_GEMV_OCC_HI : 2)
 gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restrict__ x, const int8_t *__restrict__ xq,
-            int64_t x8_pitch, const float *__restrict__ dxs, uint16_t *__restrict__ y, int M, int max_slots,
+            int64_t x8_pitch, const float *__restrict__ dxs, uint16_t *__restrict__ y, int M, int max_slots, int E,
             float *__restrict__ partial, int *__restrict__ counters) {
     constexpr int GPT = TILE / G;
     constexpr int L = B == 1 ? 1 : (1 << (B - 1));
@@ -218,16 +225,21 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
     __shared__ int s_last;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    const int64_t T = (int64_t)d.NB * d.KT, P = gridDim.x;
-    const int64_t t_begin = ((int64_t)blockIdx.x * T) / P, t_end = ((int64_t)(blockIdx.x + 1) * T) / P;
+    const int VT = d.KT + E;                       // virtual units per row block
+    const int64_t V = (int64_t)d.NB * VT, P = gridDim.x;
+    const int64_t v_begin = ((int64_t)blockIdx.x * V) / P, v_end = ((int64_t)(blockIdx.x + 1) * V) / P;
     if (threadIdx.x < 16) { s_max[threadIdx.x] = 0; s_inv[threadIdx.x] = 1.0f; }
     int8_t *ctab = nullptr;
     if constexpr (MODE == 1 && B >= 3) ctab = reinterpret_cast<int8_t *>(smem) + RT * (MAX_SUB * TILE + XS_PAD) + warp * 16 * L;
 
     bool first_slice = true;
-    for (int64_t tile = t_begin; tile < t_end;) {
-        const int nb = (int)(tile / d.KT), kb_begin = (int)(tile % d.KT);
-        const int kb_end = (int)min((int64_t)d.KT, kb_begin + (t_end - tile));
+    for (int64_t v = v_begin; v < v_end;) {
+        const int nb = (int)(v / VT);
+        const int64_t ve = min(v_end, (int64_t)(nb + 1) * VT);        // end of this CTA's units in row block nb
+        const int kb_begin = max(0, (int)(v - (int64_t)nb * VT) - E);
+        const int kb_end = max(0, (int)(ve - (int64_t)nb * VT) - E);
+        v = ve;
+        if (kb_end <= kb_begin) continue;                              // only overhead units of this row block
         float total[NT][4];
 #pragma unroll
         for (int tb = 0; tb < NT; ++tb)
@@ -358,8 +370,8 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
 
         // ---- finish this row block
         const bool whole = (kb_begin == 0 && kb_end == d.KT);
-        const int c_first = owner_of((int64_t)nb * d.KT, T, P);
-        const int n_contrib = owner_of((int64_t)(nb + 1) * d.KT - 1, T, P) - c_first + 1;
+        const int c_first = owner_of(nb, 0, d.KT, E, V, P);
+        const int n_contrib = owner_of(nb, d.KT - 1, d.KT, E, V, P) - c_first + 1;
         const int slot = (int)blockIdx.x - c_first;
         const int64_t n_lo = (int64_t)nb * TILE + warp * 16 + g;
         float *pslot = partial + ((size_t)nb * max_slots + slot) * (size_t)(M * TILE);
@@ -406,18 +418,17 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                 if (threadIdx.x == 0) counters[nb] = 0;  // leave the workspace ready for the next call
             }
         }
-        tile += (kb_end - kb_begin);
     }
 }
 
 template <int B, int G, int NT, int MODE>
 cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, const int8_t *xq, int64_t x8_pitch,
-                       const float *dxs, uint16_t *y, int M, int P, int max_slots, float *partial, int *counters,
+                       const float *dxs, uint16_t *y, int M, int P, int max_slots, int E, float *partial, int *counters,
                        cudaStream_t st) {
     constexpr int RT = 8 * NT;
     constexpr int L = B == 1 ? 1 : (1 << (B - 1));
     const int64_t T = (int64_t)d.NB * d.KT;
-    int64_t sub64 = (T + P - 1) / P + 1;
+    int64_t sub64 = (T + P - 1) / P + 2;
     if (sub64 > d.KT) sub64 = d.KT;
     if (sub64 > MAX_SUB) sub64 = MAX_SUB;
     const int sub_tiles = (int)sub64;
@@ -443,29 +454,29 @@ cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, con
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = use_pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kern, (const uint8_t *)layout, d, x, xq, x8_pitch, dxs, y, M, max_slots, partial, counters);
+    return cudaLaunchKernelEx(&cfg, kern, (const uint8_t *)layout, d, x, xq, x8_pitch, dxs, y, M, max_slots, E, partial, counters);
 }
 
 template <int B, int G>
 cudaError_t dispatch_nt_mode(const void *layout, const Dims &d, const uint16_t *x, const int8_t *xq, int64_t x8_pitch,
-                             const float *dxs, uint16_t *y, int M, int mode, int P, int max_slots, float *partial,
+                             const float *dxs, uint16_t *y, int M, int mode, int P, int max_slots, int E, float *partial,
                              int *counters, cudaStream_t st) {
     if (mode == 0) {
-        if (M <= 8) return launch_one<B, G, 1, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, partial, counters, st);
-        return launch_one<B, G, 2, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, partial, counters, st);
+        if (M <= 8) return launch_one<B, G, 1, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, E, partial, counters, st);
+        return launch_one<B, G, 2, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, E, partial, counters, st);
     }
-    if (M <= 8) return launch_one<B, G, 1, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, partial, counters, st);
-    return launch_one<B, G, 2, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, partial, counters, st);
+    if (M <= 8) return launch_one<B, G, 1, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, E, partial, counters, st);
+    return launch_one<B, G, 2, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, E, partial, counters, st);
 }
 
 template <int B>
 cudaError_t dispatch_g(const void *layout, const Dims &d, const uint16_t *x, const int8_t *xq, int64_t x8_pitch,
-                       const float *dxs, uint16_t *y, int M, int mode, int P, int max_slots, float *partial,
+                       const float *dxs, uint16_t *y, int M, int mode, int P, int max_slots, int E, float *partial,
                        int *counters, cudaStream_t st) {
     switch (d.G) {
-        case 32: return dispatch_nt_mode<B, 32>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_slots, partial, counters, st);
-        case 64: return dispatch_nt_mode<B, 64>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_slots, partial, counters, st);
-        default: return dispatch_nt_mode<B, 128>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_slots, partial, counters, st);
+        case 32: return dispatch_nt_mode<B, 32>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_slots, E, partial, counters, st);
+        case 64: return dispatch_nt_mode<B, 64>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_slots, E, partial, counters, st);
+        default: return dispatch_nt_mode<B, 128>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_slots, E, partial, counters, st);
     }
 }
 
@@ -480,9 +491,12 @@ GemvPlan gemv_plan(const Dims &d, int64_t M) {
     int64_t P = (M <= 8 && d.B <= 4 && d.G >= 64) ? 148 * CQ_GEMV_OCC_HI : 148 * 2;
     if (P > T) P = T;
     p.ctas = (int)P;
+    p.overhead = (T / P >= 6) ? 3 : 0;   // a second prologue + combine costs about three tiles of work
+    const int E = p.overhead;
+    const int64_t V = (int64_t)d.NB * (d.KT + E);
     int mx = 1;
     for (int nb = 0; nb < d.NB; ++nb) {
-        const int c = owner_of((int64_t)(nb + 1) * d.KT - 1, T, P) - owner_of((int64_t)nb * d.KT, T, P) + 1;
+        const int c = owner_of(nb, d.KT - 1, d.KT, E, V, P) - owner_of(nb, 0, d.KT, E, V, P) + 1;
         if (c > mx) mx = c;
     }
     p.max_slots = mx;
@@ -501,16 +515,16 @@ cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, ui
         cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, st);
         if (e != cudaSuccess) return e;
     }
-    const int Mi = (int)M, P = gp.ctas, ms = gp.max_slots;
+    const int Mi = (int)M, P = gp.ctas, ms = gp.max_slots, E = gp.overhead;
     switch (d.B) {
-        case 1: return dispatch_g<1>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
-        case 2: return dispatch_g<2>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
-        case 3: return dispatch_g<3>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
-        case 4: return dispatch_g<4>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
-        case 5: return dispatch_g<5>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
-        case 6: return dispatch_g<6>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
-        case 7: return dispatch_g<7>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
-        default: return dispatch_g<8>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, partial, counters, st);
+        case 1: return dispatch_g<1>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, st);
+        case 2: return dispatch_g<2>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, st);
+        case 3: return dispatch_g<3>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, st);
+        case 4: return dispatch_g<4>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, st);
+        case 5: return dispatch_g<5>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, st);
+        case 6: return dispatch_g<6>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, st);
+        case 7: return dispatch_g<7>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, st);
+        default: return dispatch_g<8>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, st);
     }
 }
 

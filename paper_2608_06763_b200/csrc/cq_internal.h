@@ -32,7 +32,7 @@ Workspace plan_workspace(const Dims &d, int64_t M, int mode);
 
 // Decomposition of the small-M path: number of CTAs (one contiguous run of tiles each) and the
 // largest number of CTAs that contribute to one 128-row block.
-struct GemvPlan { int ctas, max_slots; };
+struct GemvPlan { int ctas, max_slots, overhead; };
 GemvPlan gemv_plan(const Dims &d, int64_t M);
 
 // Small-M (M <= 16) split-K tensor-core GEMV, both activation modes.
