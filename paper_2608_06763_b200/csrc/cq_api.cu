@@ -145,14 +145,8 @@ int cq_gemm(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, in
     cudaStream_t s = (cudaStream_t)stream;
     uint8_t *ws = (uint8_t *)workspace;
     if (M <= 16) return wrap(launch_gemv(layout, d, x, y, M, mode, ws, plan, s));
-    if (mode == CQ_MODEL_DTYPE && gemm_tc_available()) return wrap(launch_gemm_tc(layout, d, x, y, M, mode, ws, plan, s));
-    // conservative route: 16 rows at a time through the small-M kernel (weights re-streamed per chunk)
-    for (int64_t m0 = 0; m0 < M; m0 += 16) {
-        const int64_t mc = (M - m0 < 16) ? (M - m0) : 16;
-        cudaError_t e = launch_gemv(layout, d, x + m0 * K, y + m0 * N, mc, mode, ws, plan, s);
-        if (e != cudaSuccess) return wrap(e);
-    }
-    return CQ_OK;
+    if (mode == CQ_MODEL_DTYPE) return wrap(launch_gemm_tc(layout, d, x, y, M, mode, ws, plan, s));
+    return wrap(launch_gemm_a8_tc(layout, d, x, y, M, ws, plan, s));
 }
 
 int cq_gemm_status(const void *workspace, size_t workspace_bytes, void *stream) {

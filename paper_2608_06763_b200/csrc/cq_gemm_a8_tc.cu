@@ -1,0 +1,325 @@
+// Large-M Dynamic-A8 GEMM on tcgen05 (Section 5.4): INT8 activation carriers x INT8 weight
+// carriers -> int32 group partials in TMEM -> fp32 rescale by s_g (and d_x / 127 at the end).
+//
+// CTA = 128 output channels x BN tokens, K walked in 128-wide blocks (one layout tile).
+//   warp 0        producer: bulk copy of the raw layout tile, TMA of the x8 tile [BN x 128] (swizzled)
+//   warp 1        TMEM allocation, tcgen05.mma kind::i8 (K = 32 per instruction); every group of
+//                 the block accumulates into its own BN columns of one of two TMEM buffers
+//   warps 2..9    decode: per group, a signed carrier table r(k) (Eq. carrier, fp32 sequence of
+//                 cq_common.cuh) for the warp's 16 rows, then one table look-up per weight into the
+//                 K-major swizzled INT8 operand tile
+//   warps 10..17  drain: tcgen05.ld of the finished int32 partials P_g, acc += s_g * P_g in fp32
+//                 registers (Eq. a8-output), so the next block's MMAs overlap; finally
+//                 y = (d_x / 127) * acc rounded to bf16
+// All mbarrier waits are bounded and report through the workspace status word.
+#include "cq_common.cuh"
+#include "cq_decode.cuh"
+#include "cq_internal.h"
+#include "cq_tc_ptx.cuh"
+
+namespace cq {
+
+namespace {
+
+using namespace tc;
+
+constexpr int A8_DEC_WARPS = 8, A8_DRAIN_WARPS = 8;
+constexpr int A8_THREADS = 32 * (2 + A8_DEC_WARPS + A8_DRAIN_WARPS);
+constexpr int A8_STAGES = 2;     // operand stages (one 128-wide k block each)
+constexpr int A8_RAW_STAGES = 2;
+constexpr int A8_SRING = 8;      // ring of per-block scale snapshots for the drain warps
+constexpr int A8_A_STAGE_BYTES = 128 * 128;
+
+struct A8Params {
+    const uint8_t *layout;
+    const float *dx;
+    uint16_t *y;
+    int *status;
+    Dims d;
+    int M;
+    int raw_stage_bytes;
+};
+
+template <int B, int G, int BN>
+__global__ void __launch_bounds__(A8_THREADS, 1)
+gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
+    constexpr int GPT = TILE / G;                 // groups per 128-wide block
+    constexpr int MPG = 4 / GPT;                  // K = 32 MMAs per group
+    constexpr int CPG = G / 16;                   // 16-wide chunks per group
+    constexpr int NCODE = 1 << B;                 // table entries (indexed by the stored code u)
+    constexpr int B_STAGE_BYTES = BN * 128;
+    constexpr uint32_t ACC_COLS = GPT * BN;       // columns of one accumulator buffer
+    constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;  // 256 or 512
+    constexpr int HALF = BN / 2;                  // columns per drain thread
+    static_assert(TMEM_COLS <= 512 && (TMEM_COLS & (TMEM_COLS - 1)) == 0, "TMEM columns");
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint8_t *sA = smem;
+    uint8_t *sB = sA + A8_STAGES * A8_A_STAGE_BYTES;
+    uint8_t *sRaw = sB + A8_STAGES * B_STAGE_BYTES;
+    int8_t *sTab = reinterpret_cast<int8_t *>(sRaw + A8_RAW_STAGES * prm.raw_stage_bytes);   // [8 warps][16 rows][NCODE]
+    float *sScale = reinterpret_cast<float *>(sTab + A8_DEC_WARPS * 16 * NCODE);              // [SRING][128][GPT]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(sScale + A8_SRING * 128 * GPT);
+    uint64_t *a_full = bars, *b_full = a_full + A8_STAGES, *st_empty = b_full + A8_STAGES;
+    uint64_t *raw_full = st_empty + A8_STAGES, *raw_empty = raw_full + A8_RAW_STAGES;
+    uint64_t *acc_full = raw_empty + A8_RAW_STAGES, *acc_empty = acc_full + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+
+    const Dims &d = prm.d;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nb = blockIdx.x, mt = blockIdx.y;
+    const int KT = d.KT;
+
+    if ((smem_u32(smem) & 1023u) != 0) {
+        if (threadIdx.x == 0) atomicCAS(prm.status, 0, 9);
+        return;
+    }
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < A8_STAGES; ++s) { mbar_init(&a_full[s], A8_DEC_WARPS); mbar_init(&b_full[s], 1); mbar_init(&st_empty[s], 1); }
+        for (int s = 0; s < A8_RAW_STAGES; ++s) { mbar_init(&raw_full[s], 1); mbar_init(&raw_empty[s], A8_DEC_WARPS); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], A8_DRAIN_WARPS); }
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ===== producer
+        if (lane == 0) {
+            const uint8_t *tiles = prm.layout + (size_t)nb * KT * (size_t)d.tile_bytes;
+            bool ok = true;
+            for (int t = 0; t < KT && ok; ++t) {
+                const int rs = t % A8_RAW_STAGES, s = t % A8_STAGES;
+                if (t >= A8_RAW_STAGES) ok = mbar_wait(&raw_empty[rs], ((t / A8_RAW_STAGES) - 1) & 1, prm.status, 11);
+                if (!ok) break;
+                mbar_arrive_expect_tx(&raw_full[rs], (uint32_t)d.tile_bytes);
+                bulk_load(sRaw + rs * prm.raw_stage_bytes, tiles + (size_t)t * d.tile_bytes, (uint32_t)d.tile_bytes, &raw_full[rs]);
+                if (t >= A8_STAGES) ok = mbar_wait(&st_empty[s], ((t / A8_STAGES) - 1) & 1, prm.status, 12);
+                if (!ok) break;
+                mbar_arrive_expect_tx(&b_full[s], B_STAGE_BYTES);
+                tma_load_2d(sB + s * B_STAGE_BYTES, &xmap, &b_full[s], t * 128, mt * BN);
+            }
+        }
+    } else if (warp == 1) {
+        // ===== MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_i8(BN);
+            bool ok = true;
+            for (int t = 0; t < KT && ok; ++t) {
+                const int s = t % A8_STAGES, ab = t & 1;
+                ok = mbar_wait(&a_full[s], (t / A8_STAGES) & 1, prm.status, 13) &&
+                     mbar_wait(&b_full[s], (t / A8_STAGES) & 1, prm.status, 14);
+                if (ok && t >= 2) ok = mbar_wait(&acc_empty[ab], ((t >> 1) - 1) & 1, prm.status, 15);
+                if (!ok) break;
+                tc_fence_after();
+                const uint64_t adesc = smem_desc_sw128(smem_u32(sA + s * A8_A_STAGE_BYTES));
+                const uint64_t bdesc = smem_desc_sw128(smem_u32(sB + s * B_STAGE_BYTES));
+#pragma unroll
+                for (int mi = 0; mi < 4; ++mi)   // four K = 32 steps, 32 bytes apart; a new group restarts the sum
+                    umma_i8(tmem_base + ab * ACC_COLS + (mi / MPG) * BN, adesc + 2 * mi, bdesc + 2 * mi, idesc, (mi % MPG) != 0);
+                umma_commit(&st_empty[s]);
+                umma_commit(&acc_full[ab]);
+            }
+        }
+    } else if (warp < 2 + A8_DEC_WARPS) {
+        // ===== decoders: warp dw owns row block dw (16 rows) of every tile
+        const int dw = warp - 2, g = lane >> 2, tq = lane & 3;
+        int8_t *tab = sTab + dw * 16 * NCODE;
+        bool ok = true;
+        for (int t = 0; t < KT && ok; ++t) {
+            const int rs = t % A8_RAW_STAGES, s = t % A8_STAGES;
+            ok = mbar_wait(&raw_full[rs], (t / A8_RAW_STAGES) & 1, prm.status, 16);
+            if (ok && t >= A8_STAGES) ok = mbar_wait(&st_empty[s], ((t / A8_STAGES) - 1) & 1, prm.status, 17);
+            if (!ok) break;
+            const uint8_t *raw = sRaw + rs * prm.raw_stage_bytes;
+            const uint8_t *rbp = raw + dw * 256 * B;
+            uint32_t w[2 * B];
+            {
+                constexpr int NFQ = (2 * B) / 4;
+#pragma unroll
+                for (int q = 0; q < NFQ; ++q) {
+                    const uint4 v = *(const uint4 *)(rbp + (q * 32 + lane) * 16);
+                    w[4 * q + 0] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+                }
+                if constexpr ((2 * B) % 4 != 0) {
+                    const uint2 v = *(const uint2 *)(rbp + NFQ * 512 + lane * 8);
+                    w[4 * NFQ + 0] = v.x; w[4 * NFQ + 1] = v.y;
+                }
+            }
+            const uint8_t *prow = raw + d.code_bytes + ((dw * 16 + g) * GPT) * 8;
+            uint8_t *a_stage = sA + s * A8_A_STAGE_BYTES;
+            uint8_t *row_lo = a_stage + (dw * 2 + 0) * 1024 + g * 128;
+            uint8_t *row_hi = a_stage + (dw * 2 + 1) * 1024 + g * 128;
+            float *sc = sScale + (size_t)(t % A8_SRING) * 128 * GPT;
+            static_for<GPT>([&](auto gc) {
+                constexpr int gi = decltype(gc)::value;
+                const uint2 p_lo = *(const uint2 *)(prow + gi * 8), p_hi = *(const uint2 *)(prow + (8 * GPT + gi) * 8);
+                if (tq == 0) {
+                    sc[(dw * 16 + g) * GPT + gi] = __uint_as_float(p_lo.x & 0x7FFFFFFFu);
+                    sc[(dw * 16 + g + 8) * GPT + gi] = __uint_as_float(p_hi.x & 0x7FFFFFFFu);
+                }
+                if constexpr (B >= 3) {
+                    // signed carrier table of this group for rows g and g + 8: index = stored code u,
+                    // u = 0 (reserved pattern) -> 0, u = 2^(B-1) + k -> sign(k) r(|k|)
+                    constexpr int Mx = (1 << (B - 1)) - 1, bias = 1 << (B - 1);
+                    __syncwarp();
+                    const __half2 ab_lo = as_h2(p_lo.y), ab_hi = as_h2(p_hi.y);
+                    const float a_lo = __low2float(ab_lo), b_lo = __high2float(ab_lo);
+                    const float a_hi = __low2float(ab_hi), b_hi = __high2float(ab_hi);
+                    int8_t *t_lo = tab + g * NCODE, *t_hi = tab + (g + 8) * NCODE;
+                    if (tq == 0) { t_lo[0] = 0; t_hi[0] = 0; }
+                    for (int i = tq; i <= Mx; i += 4) {
+                        const int r_lo = carrier_of(B, i, a_lo, b_lo), r_hi = carrier_of(B, i, a_hi, b_hi);
+                        t_lo[bias + i] = (int8_t)r_lo; t_lo[bias - i] = (int8_t)(-r_lo);
+                        t_hi[bias + i] = (int8_t)r_hi; t_hi[bias - i] = (int8_t)(-r_hi);
+                    }
+                    __syncwarp();
+                }
+                static_for<CPG>([&](auto jc) {
+                    constexpr int j = gi * CPG + decltype(jc)::value;
+                    auto carrier = [&](unsigned u, const int8_t *trow) -> uint32_t {
+                        if constexpr (B >= 3) return (uint32_t)(uint8_t)trow[u];
+                        else return (uint32_t)(uint8_t)(int8_t)(127 * signed_code(B, u));
+                    };
+                    const int8_t *t_lo = tab + g * NCODE, *t_hi = tab + (g + 8) * NCODE;
+                    const uint32_t u0 = pair_codes<B, 4 * j + 0>(w), u1 = pair_codes<B, 4 * j + 1>(w);
+                    const uint32_t u2 = pair_codes<B, 4 * j + 2>(w), u3 = pair_codes<B, 4 * j + 3>(w);
+                    const uint32_t lo = carrier(u0 & 0xFFFFu, t_lo) | (carrier(u0 >> 16, t_lo) << 8) |
+                                        (carrier(u2 & 0xFFFFu, t_lo) << 16) | (carrier(u2 >> 16, t_lo) << 24);
+                    const uint32_t hi = carrier(u1 & 0xFFFFu, t_hi) | (carrier(u1 >> 16, t_hi) << 8) |
+                                        (carrier(u3 & 0xFFFFu, t_hi) << 16) | (carrier(u3 >> 16, t_hi) << 24);
+                    // k offset inside the block: 16 j + 4 tq bytes -> 16-byte chunk j, swizzled by the row
+                    const int off = ((j ^ g) * 16) + tq * 4;
+                    *(uint32_t *)(row_lo + off) = lo;
+                    *(uint32_t *)(row_hi + off) = hi;
+                });
+            });
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(&a_full[s]); mbar_arrive(&raw_empty[rs]); }
+        }
+    } else {
+        // ===== drain warps: TMEM lane quarter warp % 4, column half (warp - 10) / 4
+        const int q4 = warp & 3, half = (warp - 2 - A8_DEC_WARPS) >> 2;
+        const int row = q4 * 32 + lane;
+        float acc[HALF];
+#pragma unroll
+        for (int i = 0; i < HALF; ++i) acc[i] = 0.0f;
+        bool ok = true;
+        for (int t = 0; t < KT && ok; ++t) {
+            const int ab = t & 1;
+            ok = mbar_wait(&acc_full[ab], (t >> 1) & 1, prm.status, 18);
+            if (!ok) break;
+            tc_fence_after();
+            const float *sc = sScale + (size_t)(t % A8_SRING) * 128 * GPT + row * GPT;
+#pragma unroll
+            for (int gi = 0; gi < GPT; ++gi) {
+                const float s = sc[gi];
+#pragma unroll
+                for (int c0 = 0; c0 < HALF; c0 += 16) {
+                    uint32_t r[16];
+                    tmem_ld16(tmem_base + ((uint32_t)(q4 * 32) << 16) + ab * ACC_COLS + gi * BN + half * HALF + c0, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) acc[c0 + i] = fmaf(s, (float)(int)r[i], acc[c0 + i]);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[ab]);
+        }
+        if (ok) {
+            const int64_t n = (int64_t)nb * TILE + row;
+            if (n < d.N) {
+#pragma unroll
+                for (int i = 0; i < HALF; ++i) {
+                    const int64_t m = (int64_t)mt * BN + half * HALF + i;
+                    if (m < prm.M) {
+                        const float v = acc[i] * (prm.dx[m] * (1.0f / 127.0f));
+                        prm.y[m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+                    }
+                }
+            }
+        }
+    }
+    if (*reinterpret_cast<volatile int *>(prm.status) != 0) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+}
+
+template <int B, int G>
+cudaError_t launch_a8(const void *layout, const Dims &d, const int8_t *x8, int64_t pitch, const float *dx, uint16_t *y,
+                      int64_t M, int *status, cudaStream_t st) {
+    constexpr int BN = G == 32 ? 64 : 128;
+    constexpr int GPT = TILE / G;
+    EncodeTiledFn enc = encode_tiled();
+    if (!enc) return cudaErrorNotSupported;
+    CUtensorMap xmap;
+    const cuuint64_t dims[2] = {(cuuint64_t)pitch, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)pitch};
+    const cuuint32_t box[2] = {128, (cuuint32_t)BN};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&xmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(x8), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+    A8Params p;
+    p.layout = (const uint8_t *)layout; p.dx = dx; p.y = y; p.status = status; p.d = d; p.M = (int)M;
+    p.raw_stage_bytes = (d.tile_bytes + 1023) / 1024 * 1024;
+    const size_t smem = (size_t)A8_STAGES * (A8_A_STAGE_BYTES + BN * 128) + (size_t)A8_RAW_STAGES * p.raw_stage_bytes +
+                        (size_t)A8_DEC_WARPS * 16 * (1 << B) + (size_t)A8_SRING * 128 * GPT * 4 + 256;
+    auto kern = gemm_a8_kernel<B, G, BN>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    dim3 grid((unsigned)d.NB, (unsigned)((M + BN - 1) / BN));
+    kern<<<grid, A8_THREADS, smem, st>>>(xmap, p);
+    return cudaGetLastError();
+}
+
+template <int B>
+cudaError_t launch_a8_b(const void *layout, const Dims &d, const int8_t *x8, int64_t pitch, const float *dx, uint16_t *y,
+                        int64_t M, int *status, cudaStream_t st) {
+    switch (d.G) {
+        case 32: return launch_a8<B, 32>(layout, d, x8, pitch, dx, y, M, status, st);
+        case 64: return launch_a8<B, 64>(layout, d, x8, pitch, dx, y, M, status, st);
+        default: return launch_a8<B, 128>(layout, d, x8, pitch, dx, y, M, status, st);
+    }
+}
+
+}  // namespace
+
+// Quantise the activations (one block per row), then run the tcgen05 INT8 GEMM on the carriers.
+cudaError_t launch_gemm_a8_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, uint8_t *ws,
+                              const Workspace &plan, cudaStream_t st) {
+    int8_t *xq = reinterpret_cast<int8_t *>(ws + plan.x8_off);
+    float *dxs = reinterpret_cast<float *>(ws + plan.dx_off);
+    int *status = reinterpret_cast<int *>(ws + plan.status_off);
+    const int64_t pitch = (int64_t)d.KT * TILE;
+    cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, st);
+    if (e != cudaSuccess) return e;
+    switch (d.B) {
+        case 1: return launch_a8_b<1>(layout, d, xq, pitch, dxs, y, M, status, st);
+        case 2: return launch_a8_b<2>(layout, d, xq, pitch, dxs, y, M, status, st);
+        case 3: return launch_a8_b<3>(layout, d, xq, pitch, dxs, y, M, status, st);
+        case 4: return launch_a8_b<4>(layout, d, xq, pitch, dxs, y, M, status, st);
+        case 5: return launch_a8_b<5>(layout, d, xq, pitch, dxs, y, M, status, st);
+        case 6: return launch_a8_b<6>(layout, d, xq, pitch, dxs, y, M, status, st);
+        case 7: return launch_a8_b<7>(layout, d, xq, pitch, dxs, y, M, status, st);
+        default: return launch_a8_b<8>(layout, d, xq, pitch, dxs, y, M, status, st);
+    }
+}
+
+}  // namespace cq

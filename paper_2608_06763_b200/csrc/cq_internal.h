@@ -42,4 +42,8 @@ cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, ui
 cudaError_t launch_gemm_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
                            uint8_t *ws, const Workspace &plan, cudaStream_t st);
 
+// Large-M Dynamic-A8 GEMM: activation quantiser, then tcgen05 kind::i8 with per-group int32 partials.
+cudaError_t launch_gemm_a8_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, uint8_t *ws,
+                              const Workspace &plan, cudaStream_t st);
+
 }  // namespace cq

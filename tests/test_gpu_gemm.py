@@ -122,3 +122,19 @@ def test_tensor_core_gemm_wide_token_tile(M):
     ws = torch.zeros(cq.cq_workspace_bytes(4, 128, M, 384, 1024, 0), dtype=torch.uint8, device="cuda")
     cq.cq_gemm(c.pw, x_to_device(x), 0, ws)
     assert cq.cq_gemm_status(ws) == 0
+
+
+@pytest.mark.parametrize("G", [32, 64, 128])
+@pytest.mark.parametrize("B", ALL_B)
+def test_tensor_core_a8_gemm_all_widths_and_groups(B, G):
+    # M = 150 runs the tcgen05 INT8 path (two token tiles, the last ragged); ragged N and K,
+    # reserved codes, a zero group, activation outlier columns
+    N, K = 200, 352 if G == 32 else 384
+    c = logical_case(N, K, B, G, seed=180 + B)
+    if B > 1:
+        c.k[5, 3:40] = -(1 << (B - 1))
+    c.s[17, 1] = 0.0
+    c = Case(c.k, c.s, c.a, c.b, B, G)
+    x = datagen.activations(150, K, seed=181, outlier_cols=0.02)
+    y, ref = run_both(c, x, cq.CQ_DYN_A8)
+    check_y(y, ref, f"a8 tc B={B} G={G}")
