@@ -2,15 +2,16 @@
 // carriers -> int32 group partials in TMEM -> fp32 rescale by s_g (and d_x / 127 at the end).
 //
 // CTA = 128 output channels x BN tokens, K walked in 128-wide blocks (one layout tile).
-//   warp 0        producer: bulk copy of the raw layout tile, TMA of the x8 tile [BN x 128] (swizzled)
-//   warp 1        TMEM allocation, tcgen05.mma kind::i8 (K = 32 per instruction); every group of
-//                 the block accumulates into its own BN columns of one of two TMEM buffers
-//   warps 2..9    decode: per group, a signed carrier table r(k) (Eq. carrier, fp32 sequence of
-//                 cq_common.cuh) for the warp's 16 rows, then one table look-up per weight into the
-//                 K-major swizzled INT8 operand tile
-//   warps 10..17  drain: tcgen05.ld of the finished int32 partials P_g, acc += s_g * P_g in fp32
-//                 registers (Eq. a8-output), so the next block's MMAs overlap; finally
-//                 y = (d_x / 127) * acc rounded to bf16
+//   warp 0       producer: bulk copy of the raw layout tile, TMA of the x8 tile [BN x 128] (swizzled)
+//   warp 1       TMEM allocation, tcgen05.mma kind::i8 (K = 32 per instruction); every group of
+//                the block accumulates into its own BN columns of one of two TMEM buffers
+//   warps 2..17  work warps, two jobs per K block, interleaved so the tensor core never waits on both:
+//                (a) decode block t: a signed carrier table r(k) per (row, group) (Eq. carrier, the
+//                    fp32 sequence of cq_common.cuh), then one table look-up per weight into the
+//                    K-major swizzled INT8 operand tile;
+//                (b) drain block t-1: tcgen05.ld of its int32 partials P_g, acc += s_g * P_g in fp32
+//                    registers (Eq. a8-output), which frees that TMEM buffer for block t+1.
+//                At the end y = (d_x / 127) * acc, rounded to bf16.
 // All mbarrier waits are bounded and report through the workspace status word.
 #include "cq_common.cuh"
 #include "cq_decode.cuh"
@@ -23,8 +24,8 @@ namespace {
 
 using namespace tc;
 
-constexpr int A8_DEC_WARPS = 8, A8_DRAIN_WARPS = 8;
-constexpr int A8_THREADS = 32 * (2 + A8_DEC_WARPS + A8_DRAIN_WARPS);
+constexpr int A8_WORK_WARPS = 16;
+constexpr int A8_THREADS = 32 * (2 + A8_WORK_WARPS);
 constexpr int A8_STAGES = 2;     // operand stages (one 128-wide k block each)
 constexpr int A8_RAW_STAGES = 2;
 constexpr int A8_SRING = 8;      // ring of per-block scale snapshots for the drain warps
@@ -40,25 +41,30 @@ struct A8Params {
     int raw_stage_bytes;
 };
 
+__device__ __forceinline__ void named_barrier_sync(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 template <int B, int G, int BN>
 __global__ void __launch_bounds__(A8_THREADS, 1)
 gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
     constexpr int GPT = TILE / G;                 // groups per 128-wide block
     constexpr int MPG = 4 / GPT;                  // K = 32 MMAs per group
-    constexpr int CPG = G / 16;                   // 16-wide chunks per group
     constexpr int NCODE = 1 << B;                 // table entries (indexed by the stored code u)
+    constexpr int Mx = B == 1 ? 1 : (1 << (B - 1)) - 1;
     constexpr int B_STAGE_BYTES = BN * 128;
     constexpr uint32_t ACC_COLS = GPT * BN;       // columns of one accumulator buffer
-    constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;  // 256 or 512
-    constexpr int HALF = BN / 2;                  // columns per drain thread
+    constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;  // 512
+    constexpr int QCOLS = BN / 4;                 // columns per work thread in the drain
     static_assert(TMEM_COLS <= 512 && (TMEM_COLS & (TMEM_COLS - 1)) == 0, "TMEM columns");
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t *sA = smem;
     uint8_t *sB = sA + A8_STAGES * A8_A_STAGE_BYTES;
     uint8_t *sRaw = sB + A8_STAGES * B_STAGE_BYTES;
-    int8_t *sTab = reinterpret_cast<int8_t *>(sRaw + A8_RAW_STAGES * prm.raw_stage_bytes);   // [8 warps][16 rows][NCODE]
-    float *sScale = reinterpret_cast<float *>(sTab + A8_DEC_WARPS * 16 * NCODE);              // [SRING][128][GPT]
-    uint64_t *bars = reinterpret_cast<uint64_t *>(sScale + A8_SRING * 128 * GPT);
+    int8_t *sTab = reinterpret_cast<int8_t *>(sRaw + A8_RAW_STAGES * prm.raw_stage_bytes);   // [8 row blocks][2][16 rows][NCODE]
+    float *sScale = reinterpret_cast<float *>(sTab + 8 * 2 * 16 * NCODE);                      // [SRING][128][GPT]
+    float *sT = sScale + A8_SRING * 128 * GPT;                                                 // t_i = i / M, i = 0..127
+    uint64_t *bars = reinterpret_cast<uint64_t *>(sT + 128);
     uint64_t *a_full = bars, *b_full = a_full + A8_STAGES, *st_empty = b_full + A8_STAGES;
     uint64_t *raw_full = st_empty + A8_STAGES, *raw_empty = raw_full + A8_RAW_STAGES;
     uint64_t *acc_full = raw_empty + A8_RAW_STAGES, *acc_empty = acc_full + 2;
@@ -74,11 +80,12 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
         return;
     }
     if (threadIdx.x == 0) {
-        for (int s = 0; s < A8_STAGES; ++s) { mbar_init(&a_full[s], A8_DEC_WARPS); mbar_init(&b_full[s], 1); mbar_init(&st_empty[s], 1); }
-        for (int s = 0; s < A8_RAW_STAGES; ++s) { mbar_init(&raw_full[s], 1); mbar_init(&raw_empty[s], A8_DEC_WARPS); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], A8_DRAIN_WARPS); }
+        for (int s = 0; s < A8_STAGES; ++s) { mbar_init(&a_full[s], A8_WORK_WARPS); mbar_init(&b_full[s], 1); mbar_init(&st_empty[s], 1); }
+        for (int s = 0; s < A8_RAW_STAGES; ++s) { mbar_init(&raw_full[s], 1); mbar_init(&raw_empty[s], A8_WORK_WARPS); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], A8_WORK_WARPS); }
         fence_barrier_init();
     }
+    if (threadIdx.x < 128) sT[threadIdx.x] = __fdiv_rn((float)threadIdx.x, (float)Mx);  // the pinned t = i / M
     if (warp == 1) {
         tmem_alloc(tmem_slot, TMEM_COLS);
         tmem_relinquish();
@@ -126,119 +133,141 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
                 umma_commit(&acc_full[ab]);
             }
         }
-    } else if (warp < 2 + A8_DEC_WARPS) {
-        // ===== decoders: warp dw owns row block dw (16 rows) of every tile
-        const int dw = warp - 2, g = lane >> 2, tq = lane & 3;
-        int8_t *tab = sTab + dw * 16 * NCODE;
-        bool ok = true;
-        for (int t = 0; t < KT && ok; ++t) {
-            const int rs = t % A8_RAW_STAGES, s = t % A8_STAGES;
-            ok = mbar_wait(&raw_full[rs], (t / A8_RAW_STAGES) & 1, prm.status, 16);
-            if (ok && t >= A8_STAGES) ok = mbar_wait(&st_empty[s], ((t / A8_STAGES) - 1) & 1, prm.status, 17);
-            if (!ok) break;
-            const uint8_t *raw = sRaw + rs * prm.raw_stage_bytes;
-            const uint8_t *rbp = raw + dw * 256 * B;
-            uint32_t w[2 * B];
-            {
-                constexpr int NFQ = (2 * B) / 4;
-#pragma unroll
-                for (int q = 0; q < NFQ; ++q) {
-                    const uint4 v = *(const uint4 *)(rbp + (q * 32 + lane) * 16);
-                    w[4 * q + 0] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
-                }
-                if constexpr ((2 * B) % 4 != 0) {
-                    const uint2 v = *(const uint2 *)(rbp + NFQ * 512 + lane * 8);
-                    w[4 * NFQ + 0] = v.x; w[4 * NFQ + 1] = v.y;
-                }
-            }
-            const uint8_t *prow = raw + d.code_bytes + ((dw * 16 + g) * GPT) * 8;
-            uint8_t *a_stage = sA + s * A8_A_STAGE_BYTES;
-            uint8_t *row_lo = a_stage + (dw * 2 + 0) * 1024 + g * 128;
-            uint8_t *row_hi = a_stage + (dw * 2 + 1) * 1024 + g * 128;
-            float *sc = sScale + (size_t)(t % A8_SRING) * 128 * GPT;
-            static_for<GPT>([&](auto gc) {
-                constexpr int gi = decltype(gc)::value;
-                const uint2 p_lo = *(const uint2 *)(prow + gi * 8), p_hi = *(const uint2 *)(prow + (8 * GPT + gi) * 8);
-                if (tq == 0) {
-                    sc[(dw * 16 + g) * GPT + gi] = __uint_as_float(p_lo.x & 0x7FFFFFFFu);
-                    sc[(dw * 16 + g + 8) * GPT + gi] = __uint_as_float(p_hi.x & 0x7FFFFFFFu);
-                }
-                if constexpr (B >= 3) {
-                    // signed carrier table of this group for rows g and g + 8: index = stored code u,
-                    // u = 0 (reserved pattern) -> 0, u = 2^(B-1) + k -> sign(k) r(|k|)
-                    constexpr int Mx = (1 << (B - 1)) - 1, bias = 1 << (B - 1);
-                    __syncwarp();
-                    const __half2 ab_lo = as_h2(p_lo.y), ab_hi = as_h2(p_hi.y);
-                    const float a_lo = __low2float(ab_lo), b_lo = __high2float(ab_lo);
-                    const float a_hi = __low2float(ab_hi), b_hi = __high2float(ab_hi);
-                    int8_t *t_lo = tab + g * NCODE, *t_hi = tab + (g + 8) * NCODE;
-                    if (tq == 0) { t_lo[0] = 0; t_hi[0] = 0; }
-                    for (int i = tq; i <= Mx; i += 4) {
-                        const int r_lo = carrier_of(B, i, a_lo, b_lo), r_hi = carrier_of(B, i, a_hi, b_hi);
-                        t_lo[bias + i] = (int8_t)r_lo; t_lo[bias - i] = (int8_t)(-r_lo);
-                        t_hi[bias + i] = (int8_t)r_hi; t_hi[bias - i] = (int8_t)(-r_hi);
-                    }
-                    __syncwarp();
-                }
-                static_for<CPG>([&](auto jc) {
-                    constexpr int j = gi * CPG + decltype(jc)::value;
-                    auto carrier = [&](unsigned u, const int8_t *trow) -> uint32_t {
-                        if constexpr (B >= 3) return (uint32_t)(uint8_t)trow[u];
-                        else return (uint32_t)(uint8_t)(int8_t)(127 * signed_code(B, u));
-                    };
-                    const int8_t *t_lo = tab + g * NCODE, *t_hi = tab + (g + 8) * NCODE;
-                    const uint32_t u0 = pair_codes<B, 4 * j + 0>(w), u1 = pair_codes<B, 4 * j + 1>(w);
-                    const uint32_t u2 = pair_codes<B, 4 * j + 2>(w), u3 = pair_codes<B, 4 * j + 3>(w);
-                    const uint32_t lo = carrier(u0 & 0xFFFFu, t_lo) | (carrier(u0 >> 16, t_lo) << 8) |
-                                        (carrier(u2 & 0xFFFFu, t_lo) << 16) | (carrier(u2 >> 16, t_lo) << 24);
-                    const uint32_t hi = carrier(u1 & 0xFFFFu, t_hi) | (carrier(u1 >> 16, t_hi) << 8) |
-                                        (carrier(u3 & 0xFFFFu, t_hi) << 16) | (carrier(u3 >> 16, t_hi) << 24);
-                    // k offset inside the block: 16 j + 4 tq bytes -> 16-byte chunk j, swizzled by the row
-                    const int off = ((j ^ g) * 16) + tq * 4;
-                    *(uint32_t *)(row_lo + off) = lo;
-                    *(uint32_t *)(row_hi + off) = hi;
-                });
-            });
-            fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) { mbar_arrive(&a_full[s]); mbar_arrive(&raw_empty[rs]); }
-        }
     } else {
-        // ===== drain warps: TMEM lane quarter warp % 4, column half (warp - 10) / 4
-        const int q4 = warp & 3, half = (warp - 2 - A8_DEC_WARPS) >> 2;
-        const int row = q4 * 32 + lane;
-        float acc[HALF];
+        // ===== work warps.  Decode: warp dw owns row block dw / 2 and the 64-wide half dw % 2 of every
+        // block.  Drain: TMEM lane quarter warp % 4, column quarter dw / 4.
+        const int dw = warp - 2, g = lane >> 2, tq = lane & 3;
+        const int rb = dw >> 1, jh = dw & 1;
+        const int q4 = warp & 3, cq4 = dw >> 2;
+        const int drow = q4 * 32 + lane;
+        int8_t *tab = sTab + (rb * 2 + (G == 128 ? 0 : jh)) * 16 * NCODE;   // G = 128: the two halves share one table
+        float acc[QCOLS];
 #pragma unroll
-        for (int i = 0; i < HALF; ++i) acc[i] = 0.0f;
+        for (int i = 0; i < QCOLS; ++i) acc[i] = 0.0f;
         bool ok = true;
-        for (int t = 0; t < KT && ok; ++t) {
-            const int ab = t & 1;
-            ok = mbar_wait(&acc_full[ab], (t >> 1) & 1, prm.status, 18);
-            if (!ok) break;
-            tc_fence_after();
-            const float *sc = sScale + (size_t)(t % A8_SRING) * 128 * GPT + row * GPT;
+        for (int t = 0; t <= KT && ok; ++t) {
+            if (t < KT) {
+                // ---------------- (a) decode block t
+                const int rs = t % A8_RAW_STAGES, s = t % A8_STAGES;
+                ok = mbar_wait(&raw_full[rs], (t / A8_RAW_STAGES) & 1, prm.status, 16);
+                if (ok && t >= A8_STAGES) ok = mbar_wait(&st_empty[s], ((t / A8_STAGES) - 1) & 1, prm.status, 17);
+                if (!ok) break;
+                const uint8_t *raw = sRaw + rs * prm.raw_stage_bytes;
+                const uint8_t *rbp = raw + rb * 256 * B;
+                uint32_t w[2 * B];
+                {
+                    constexpr int NFQ = (2 * B) / 4;
 #pragma unroll
-            for (int gi = 0; gi < GPT; ++gi) {
-                const float s = sc[gi];
-#pragma unroll
-                for (int c0 = 0; c0 < HALF; c0 += 16) {
-                    uint32_t r[16];
-                    tmem_ld16(tmem_base + ((uint32_t)(q4 * 32) << 16) + ab * ACC_COLS + gi * BN + half * HALF + c0, r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) acc[c0 + i] = fmaf(s, (float)(int)r[i], acc[c0 + i]);
+                    for (int q = 0; q < NFQ; ++q) {
+                        const uint4 v = *(const uint4 *)(rbp + (q * 32 + lane) * 16);
+                        w[4 * q + 0] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+                    }
+                    if constexpr ((2 * B) % 4 != 0) {
+                        const uint2 v = *(const uint2 *)(rbp + NFQ * 512 + lane * 8);
+                        w[4 * NFQ + 0] = v.x; w[4 * NFQ + 1] = v.y;
+                    }
                 }
+                const uint8_t *prow = raw + d.code_bytes + ((rb * 16 + g) * GPT) * 8;
+                uint8_t *a_stage = sA + s * A8_A_STAGE_BYTES;
+                uint8_t *row_lo = a_stage + (rb * 2 + 0) * 1024 + g * 128;
+                uint8_t *row_hi = a_stage + (rb * 2 + 1) * 1024 + g * 128;
+                float *sc = sScale + (size_t)(t % A8_SRING) * 128 * GPT;
+                constexpr int GH = GPT >= 2 ? GPT / 2 : 1;   // groups this warp's 64-wide half touches
+                constexpr int CPGH = 4 / GH;                 // 16-wide chunks of the half per such group
+                auto do_half = [&](auto jhc) {
+                    constexpr int JH = decltype(jhc)::value;
+                    static_for<GH>([&](auto gc) {
+                        constexpr int gi = (GPT >= 2) ? JH * GH + decltype(gc)::value : 0;
+                        const uint2 p_lo = *(const uint2 *)(prow + gi * 8), p_hi = *(const uint2 *)(prow + (8 * GPT + gi) * 8);
+                        if (tq == 0 && (G != 128 || JH == 0)) {
+                            sc[(rb * 16 + g) * GPT + gi] = __uint_as_float(p_lo.x & 0x7FFFFFFFu);
+                            sc[(rb * 16 + g + 8) * GPT + gi] = __uint_as_float(p_hi.x & 0x7FFFFFFFu);
+                        }
+                        if constexpr (B >= 3) {
+                            // signed carrier table: index = stored code u; u = 0 (reserved) -> 0,
+                            // u = 2^(B-1) + k -> sign(k) r(|k|).  With G = 128 the two warps of a row block
+                            // build eight rows each and meet at a 64-thread barrier.
+                            constexpr int bias = 1 << (B - 1);
+                            if constexpr (G == 128) named_barrier_sync(1 + rb, 64); else __syncwarp();
+                            auto build_row = [&](int row, uint32_t abbits) {
+                                const __half2 ab = as_h2(abbits);
+                                const float a = __low2float(ab), b = __high2float(ab);
+                                const float c = __fsub_rn(__fsub_rn(1.0f, a), b);
+                                int8_t *tr = tab + row * NCODE;
+                                if (tq == 0) tr[0] = 0;
+                                for (int i = tq; i <= Mx; i += 4) {
+                                    const float tt = sT[i];
+                                    const float q = __fmul_rn(tt, fmaf(tt, fmaf(tt, c, b), a));
+                                    int r = __float2int_rn(__fmul_rn(127.0f, q));
+                                    r = min(max(r, 0), 127);
+                                    tr[bias + i] = (int8_t)r;
+                                    tr[bias - i] = (int8_t)(-r);
+                                }
+                            };
+                            if constexpr (G == 128) {
+                                if (JH == 0) build_row(g, p_lo.y); else build_row(g + 8, p_hi.y);
+                                named_barrier_sync(1 + rb, 64);
+                            } else {
+                                build_row(g, p_lo.y);
+                                build_row(g + 8, p_hi.y);
+                                __syncwarp();
+                            }
+                        }
+                        static_for<CPGH>([&](auto jc) {
+                            constexpr int j = 4 * JH + decltype(gc)::value * CPGH + decltype(jc)::value;
+                            auto carrier = [&](unsigned u, const int8_t *trow) -> uint32_t {
+                                if constexpr (B >= 3) return (uint32_t)(uint8_t)trow[u];
+                                else return (uint32_t)(uint8_t)(int8_t)(127 * signed_code(B, u));
+                            };
+                            const int8_t *t_lo = tab + g * NCODE, *t_hi = tab + (g + 8) * NCODE;
+                            const uint32_t u0 = pair_codes<B, 4 * j + 0>(w), u1 = pair_codes<B, 4 * j + 1>(w);
+                            const uint32_t u2 = pair_codes<B, 4 * j + 2>(w), u3 = pair_codes<B, 4 * j + 3>(w);
+                            const uint32_t lo = carrier(u0 & 0xFFFFu, t_lo) | (carrier(u0 >> 16, t_lo) << 8) |
+                                                (carrier(u2 & 0xFFFFu, t_lo) << 16) | (carrier(u2 >> 16, t_lo) << 24);
+                            const uint32_t hi = carrier(u1 & 0xFFFFu, t_hi) | (carrier(u1 >> 16, t_hi) << 8) |
+                                                (carrier(u3 & 0xFFFFu, t_hi) << 16) | (carrier(u3 >> 16, t_hi) << 24);
+                            // k offset inside the block: 16 j + 4 tq bytes -> 16-byte chunk j, swizzled by the row
+                            const int off = ((j ^ g) * 16) + tq * 4;
+                            *(uint32_t *)(row_lo + off) = lo;
+                            *(uint32_t *)(row_hi + off) = hi;
+                        });
+                    });
+                };
+                if (jh == 0) do_half(std::integral_constant<int, 0>{}); else do_half(std::integral_constant<int, 1>{});
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) { mbar_arrive(&a_full[s]); mbar_arrive(&raw_empty[rs]); }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[ab]);
+            if (t >= 1) {
+                // ---------------- (b) drain block t - 1
+                const int td = t - 1, ab = td & 1;
+                ok = mbar_wait(&acc_full[ab], (td >> 1) & 1, prm.status, 18);
+                if (!ok) break;
+                tc_fence_after();
+                const float *scd = sScale + (size_t)(td % A8_SRING) * 128 * GPT + drow * GPT;
+#pragma unroll
+                for (int gi = 0; gi < GPT; ++gi) {
+                    const float sg = scd[gi];
+#pragma unroll
+                    for (int c0 = 0; c0 < QCOLS; c0 += 16) {
+                        uint32_t r[16];
+                        tmem_ld16(tmem_base + ((uint32_t)(q4 * 32) << 16) + ab * ACC_COLS + gi * BN + cq4 * QCOLS + c0, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) acc[c0 + i] = fmaf(sg, (float)(int)r[i], acc[c0 + i]);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[ab]);
+            }
         }
         if (ok) {
-            const int64_t n = (int64_t)nb * TILE + row;
+            const int64_t n = (int64_t)nb * TILE + drow;
             if (n < d.N) {
 #pragma unroll
-                for (int i = 0; i < HALF; ++i) {
-                    const int64_t m = (int64_t)mt * BN + half * HALF + i;
+                for (int i = 0; i < QCOLS; ++i) {
+                    const int64_t m = (int64_t)mt * BN + cq4 * QCOLS + i;
                     if (m < prm.M) {
                         const float v = acc[i] * (prm.dx[m] * (1.0f / 127.0f));
                         prm.y[m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
@@ -259,8 +288,8 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
 template <int B, int G>
 cudaError_t launch_a8(const void *layout, const Dims &d, const int8_t *x8, int64_t pitch, const float *dx, uint16_t *y,
                       int64_t M, int *status, cudaStream_t st) {
-    constexpr int BN = G == 32 ? 64 : 128;
     constexpr int GPT = TILE / G;
+    constexpr int BN = 256 / GPT;   // two accumulator buffers of GPT x BN columns fill the 512 TMEM columns
     EncodeTiledFn enc = encode_tiled();
     if (!enc) return cudaErrorNotSupported;
     CUtensorMap xmap;
@@ -276,7 +305,7 @@ cudaError_t launch_a8(const void *layout, const Dims &d, const int8_t *x8, int64
     p.layout = (const uint8_t *)layout; p.dx = dx; p.y = y; p.status = status; p.d = d; p.M = (int)M;
     p.raw_stage_bytes = (d.tile_bytes + 1023) / 1024 * 1024;
     const size_t smem = (size_t)A8_STAGES * (A8_A_STAGE_BYTES + BN * 128) + (size_t)A8_RAW_STAGES * p.raw_stage_bytes +
-                        (size_t)A8_DEC_WARPS * 16 * (1 << B) + (size_t)A8_SRING * 128 * GPT * 4 + 256;
+                        (size_t)8 * 2 * 16 * (1 << B) + (size_t)A8_SRING * 128 * GPT * 4 + 512 + 256;
     auto kern = gemm_a8_kernel<B, G, BN>;
     static bool attr_done = false;
     if (!attr_done) {
