@@ -172,7 +172,16 @@ def extra_suites(torch, cq, datagen, stream, peaks):
             gemm.append({"shape": name, "K": K, "N": N, "M": M, "B": B, "G": 128, "mode": "model_dtype",
                          "ms": round(ms, 4), "tflops": round(tf, 1),
                          "frac_of_measured_bf16_burst": round(tf / peaks["bf16_tflops"], 4)})
-            del pw, ws
+            ws8 = torch.zeros(cq.cq_workspace_bytes(B, 128, M, N, K, 1), dtype=torch.uint8, device="cuda")
+            for _ in range(2):
+                cq.cq_gemm(pw, x, cq.CQ_DYN_A8, ws8, y)
+            ms8 = time_graph(torch, stream, lambda i: cq.cq_gemm(pw, x, cq.CQ_DYN_A8, ws8, y), 3)
+            tops = 2.0 * M * N * K / (ms8 * 1e-3) / 1e12
+            gemm.append({"shape": name, "K": K, "N": N, "M": M, "B": B, "G": 128, "mode": "dyn_a8",
+                         "ms": round(ms8, 4), "tops": round(tops, 1),
+                         "frac_of_nominal_int8_dense_4500": round(tops / 4500.0, 4),
+                         "note": "includes the activation quantiser launch"})
+            del pw, ws, ws8
         del x, y
         torch.cuda.empty_cache()
     out["gemm_prefill"] = gemm
