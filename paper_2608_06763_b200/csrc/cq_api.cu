@@ -21,8 +21,14 @@ Workspace plan_workspace(const Dims &d, int64_t M, int mode) {
     const GemvPlan gp = gemv_plan(d, Mc);
     size_t off = 0;
     w.status_off = off; off += 256;  // first, so cq_gemm_status finds it without knowing the problem
-    w.counters_off = off; w.counters_bytes = align_up((size_t)d.NB * 4, 256); off += w.counters_bytes;
-    w.partial_off = off; w.partial_bytes = align_up((size_t)d.NB * gp.max_slots * Mc * TILE * 4, 256); off += w.partial_bytes;
+    // arrival counters: one per 128-row block (small M) or per output tile (split-K GEMM)
+    const int64_t bnt = gemm_tc_token_tile(M);
+    const int sk = (M > 16 && mode == CQ_MODEL_DTYPE) ? gemm_tc_split_k(d, M) : 1;
+    const size_t n_ctr = (size_t)d.NB * (M > 16 ? (size_t)((M + bnt - 1) / bnt) : 1);
+    w.counters_off = off; w.counters_bytes = align_up(n_ctr * 4, 256); off += w.counters_bytes;
+    size_t part = (size_t)d.NB * gp.max_slots * Mc * TILE * 4;
+    if (sk > 1) { const size_t p2 = (size_t)sk * M * d.NB * TILE * 4; if (p2 > part) part = p2; }
+    w.partial_off = off; w.partial_bytes = align_up(part, 256); off += w.partial_bytes;
     if (mode == CQ_DYN_A8) {
         w.x8_off = off; w.x8_bytes = align_up((size_t)(M + 127) / 128 * 128 * Kp, 256); off += w.x8_bytes;
         w.dx_off = off; w.dx_bytes = align_up((size_t)M * 4, 256); off += w.dx_bytes;

@@ -24,6 +24,19 @@ namespace cq {
 
 int gemm_tc_available() { return 1; }
 
+// Token tile of the model-dtype GEMM for M rows, and its split-K factor: when the output tiles
+// alone would leave most of the 148 SMs idle, the K range is cut so that about one CTA per SM runs.
+int gemm_tc_token_tile(int64_t M) { return M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : M <= 256 ? 256 : 512; }
+int gemm_tc_split_k(const Dims &d, int64_t M) {
+    const int64_t bnt = gemm_tc_token_tile(M);
+    const int64_t ctas = (int64_t)d.NB * ((M + bnt - 1) / bnt);
+    if (ctas >= 100 || M > 256) return 1;   // the combine of a large token tile costs more than the idle SMs
+    int64_t sk = 148 / ctas;
+    if (sk > 8) sk = 8;
+    if (sk > d.KT / 4) sk = d.KT / 4;   // at least four layout tiles per slice
+    return sk < 1 ? 1 : (int)sk;
+}
+
 namespace {
 
 using namespace tc;
@@ -53,6 +66,8 @@ struct TcParams {
     Dims d;
     int M;
     int raw_stage_bytes;  // tile_bytes rounded up to 1024
+    float *partial;       // split-K: fp32 partial sums [SK][M][Np]
+    int *counters;        // split-K: arrival counters, one per (row block, token tile)
 };
 
 // ---------------------------------------------------------------- the kernel (model dtype)
@@ -81,7 +96,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
     const Dims &d = prm.d;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nb = blockIdx.x, mt = blockIdx.y;
-    const int KT = d.KT;            // layout tiles along K
+    // split-K: blockIdx.z takes the layout tiles [kt0, kt0 + KT) of the K range
+    const int kt0 = (int)(((int64_t)d.KT * blockIdx.z) / gridDim.z);
+    const int KT = (int)(((int64_t)d.KT * (blockIdx.z + 1)) / gridDim.z) - kt0;
     const int NKB = 2 * KT;         // 64-wide k blocks
 
     if ((smem_u32(smem) & 1023u) != 0) {  // cannot happen with the alignment attribute; never run misaligned
@@ -106,7 +123,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
     if (warp == 0) {
         // ===== producer
         if (lane == 0) {
-            const uint8_t *tiles = prm.layout + (size_t)nb * KT * (size_t)d.tile_bytes;
+            const uint8_t *tiles = prm.layout + ((size_t)nb * d.KT + kt0) * (size_t)d.tile_bytes;
             bool ok = true;
             for (int kb = 0; kb < NKB && ok; ++kb) {
                 if ((kb & 1) == 0) {
@@ -122,7 +139,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                 mbar_arrive_expect_tx(&b_full[s], B_STAGE_BYTES);
 #pragma unroll
                 for (int a = 0; a < NACC; ++a)
-                    tma_load_2d(sB + s * B_STAGE_BYTES + a * B_TILE_BYTES, &xmap, &b_full[s], kb * 64, mt * BNT + a * BN);
+                    tma_load_2d(sB + s * B_STAGE_BYTES + a * B_TILE_BYTES, &xmap, &b_full[s], (2 * kt0 + kb) * 64, mt * BNT + a * BN);
             }
         }
     } else if (warp == 1) {
@@ -232,11 +249,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                 uint32_t r[32];
                 tmem_ld32(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)c0, r);
                 tmem_ld_wait();
-                if (n < d.N) {
+                if (n < d.N || gridDim.z > 1) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         const int64_t m = (int64_t)mt * BNT + c0 + i;
-                        if (m < prm.M) prm.y[m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(r[i])));
+                        if (m < prm.M) {
+                            if (gridDim.z == 1) prm.y[m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(r[i])));
+                            else prm.partial[((size_t)blockIdx.z * prm.M + m) * ((size_t)d.NB * TILE) + n] = __uint_as_float(r[i]);
+                        }
                     }
                 }
             }
@@ -250,12 +270,58 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+    if (gridDim.z > 1) {
+        // split-K combine: the last CTA of this output tile to arrive adds the slices in slice order.
+        // The barrier above ordered the CTA's partial stores before thread 0's release.
+        volatile int *s_last_p = reinterpret_cast<volatile int *>(tmem_slot + 1);   // scratch word after the TMEM slot
+        int *ctr = prm.counters + (nb * gridDim.y + mt);
+        if (threadIdx.x == 0) {
+            int old;
+            asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(ctr) : "memory");
+            *s_last_p = (old == (int)gridDim.z - 1);
+        }
+        __syncthreads();
+        if (*s_last_p) {
+            const size_t Np = (size_t)d.NB * TILE;
+            // each thread takes four consecutive channels of one token at a time (128-bit loads), two such
+            // quads per step, all loads issued before the sums
+            constexpr int QUADS = BNT * TILE / 4;
+            for (int base = threadIdx.x; base < QUADS; base += 2 * TC_THREADS) {
+                float4 v[2][8];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int qd = base + u * TC_THREADS;
+                    const int64_t m = (int64_t)mt * BNT + qd / (TILE / 4), n = (int64_t)nb * TILE + (qd % (TILE / 4)) * 4;
+                    const bool live = qd < QUADS && m < prm.M;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        v[u][q] = (live && q < (int)gridDim.z)
+                                      ? __ldcg(reinterpret_cast<const float4 *>(prm.partial + ((size_t)q * prm.M + m) * Np + n))
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int qd = base + u * TC_THREADS;
+                    const int64_t m = (int64_t)mt * BNT + qd / (TILE / 4), n = (int64_t)nb * TILE + (qd % (TILE / 4)) * 4;
+                    if (qd >= QUADS || m >= prm.M) continue;
+                    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) { sum.x += v[u][q].x; sum.y += v[u][q].y; sum.z += v[u][q].z; sum.w += v[u][q].w; }  // slice order
+                    const float o[4] = {sum.x, sum.y, sum.z, sum.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (n + e < d.N) prm.y[m * d.N + n + e] = __bfloat16_as_ushort(__float2bfloat16_rn(o[e]));
+                }
+            }
+            if (threadIdx.x == 0) *ctr = 0;  // leave the workspace ready for the next call
+        }
+    }
 }
 
 // ---------------------------------------------------------------- host side
 template <int B, int G, int BN, int NACC>
 cudaError_t launch_bn(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int *status,
-                      cudaStream_t st) {
+                      float *partial, int *counters, cudaStream_t st) {
     EncodeTiledFn enc = encode_tiled();
     if (!enc) return cudaErrorNotSupported;
     CUtensorMap xmap;
@@ -279,28 +345,29 @@ cudaError_t launch_bn(const void *layout, const Dims &d, const uint16_t *x, uint
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    dim3 grid((unsigned)d.NB, (unsigned)((M + BN * NACC - 1) / (BN * NACC)));
+    p.partial = partial; p.counters = counters;
+    dim3 grid((unsigned)d.NB, (unsigned)((M + BN * NACC - 1) / (BN * NACC)), (unsigned)gemm_tc_split_k(d, M));
     kern<<<grid, TC_THREADS, smem, st>>>(xmap, p);
     return cudaGetLastError();
 }
 
 template <int B, int G>
 cudaError_t launch_g(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int *status,
-                     cudaStream_t st) {
-    if (M <= 32) return launch_bn<B, G, 32, 1>(layout, d, x, y, M, status, st);
-    if (M <= 64) return launch_bn<B, G, 64, 1>(layout, d, x, y, M, status, st);
-    if (M <= 128) return launch_bn<B, G, 128, 1>(layout, d, x, y, M, status, st);
-    if (M <= 256) return launch_bn<B, G, 256, 1>(layout, d, x, y, M, status, st);
-    return launch_bn<B, G, 256, 2>(layout, d, x, y, M, status, st);
+                     float *partial, int *counters, cudaStream_t st) {
+    if (M <= 32) return launch_bn<B, G, 32, 1>(layout, d, x, y, M, status, partial, counters, st);
+    if (M <= 64) return launch_bn<B, G, 64, 1>(layout, d, x, y, M, status, partial, counters, st);
+    if (M <= 128) return launch_bn<B, G, 128, 1>(layout, d, x, y, M, status, partial, counters, st);
+    if (M <= 256) return launch_bn<B, G, 256, 1>(layout, d, x, y, M, status, partial, counters, st);
+    return launch_bn<B, G, 256, 2>(layout, d, x, y, M, status, partial, counters, st);
 }
 
 template <int B>
 cudaError_t launch_b(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int *status,
-                     cudaStream_t st) {
+                     float *partial, int *counters, cudaStream_t st) {
     switch (d.G) {
-        case 32: return launch_g<B, 32>(layout, d, x, y, M, status, st);
-        case 64: return launch_g<B, 64>(layout, d, x, y, M, status, st);
-        default: return launch_g<B, 128>(layout, d, x, y, M, status, st);
+        case 32: return launch_g<B, 32>(layout, d, x, y, M, status, partial, counters, st);
+        case 64: return launch_g<B, 64>(layout, d, x, y, M, status, partial, counters, st);
+        default: return launch_g<B, 128>(layout, d, x, y, M, status, partial, counters, st);
     }
 }
 
@@ -310,15 +377,17 @@ cudaError_t launch_gemm_tc(const void *layout, const Dims &d, const uint16_t *x,
                            uint8_t *ws, const Workspace &plan, cudaStream_t st) {
     if (mode != 0) return cudaErrorNotSupported;
     int *status = reinterpret_cast<int *>(ws + plan.status_off);
+    float *partial = reinterpret_cast<float *>(ws + plan.partial_off);
+    int *counters = reinterpret_cast<int *>(ws + plan.counters_off);
     switch (d.B) {
-        case 1: return launch_b<1>(layout, d, x, y, M, status, st);
-        case 2: return launch_b<2>(layout, d, x, y, M, status, st);
-        case 3: return launch_b<3>(layout, d, x, y, M, status, st);
-        case 4: return launch_b<4>(layout, d, x, y, M, status, st);
-        case 5: return launch_b<5>(layout, d, x, y, M, status, st);
-        case 6: return launch_b<6>(layout, d, x, y, M, status, st);
-        case 7: return launch_b<7>(layout, d, x, y, M, status, st);
-        default: return launch_b<8>(layout, d, x, y, M, status, st);
+        case 1: return launch_b<1>(layout, d, x, y, M, status, partial, counters, st);
+        case 2: return launch_b<2>(layout, d, x, y, M, status, partial, counters, st);
+        case 3: return launch_b<3>(layout, d, x, y, M, status, partial, counters, st);
+        case 4: return launch_b<4>(layout, d, x, y, M, status, partial, counters, st);
+        case 5: return launch_b<5>(layout, d, x, y, M, status, partial, counters, st);
+        case 6: return launch_b<6>(layout, d, x, y, M, status, partial, counters, st);
+        case 7: return launch_b<7>(layout, d, x, y, M, status, partial, counters, st);
+        default: return launch_b<8>(layout, d, x, y, M, status, partial, counters, st);
     }
 }
 
