@@ -212,6 +212,27 @@ def extra_suites(torch, cq, datagen, stream, peaks):
                                   "us_a8": round(t[1] * 1e3, 2), "model_over_a8": round(t[0] / t[1], 3)})
         del pws, copies
         torch.cuda.empty_cache()
+    # ---- the paper's own kernel-measurement shapes (Section 6.3: G512, W2/W5/W8, M in {1,16,64,256}),
+    # so B200 numbers can sit beside its H200 table (context only)
+    paper = []
+    for N, K in ((3584, 3072), (6144, 3584)):
+        for B in (2, 5, 8):
+            pw = make_packed_cuda(cq, datagen, N, K, B, 512, 5)
+            cp = [pw] + [cq.PackedWeights(pw.layout.clone(), B, 512, N, K) for _ in range(int(np.ceil(2 * L2_BYTES / pw.layout.numel())))]
+            for M in (1, 16, 64, 256):
+                x = datagen.activations_cuda(M, K, seed=5)
+                y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+                t = {}
+                for mode in (cq.CQ_MODEL_DTYPE, cq.CQ_DYN_A8):
+                    ws = torch.zeros(cq.cq_workspace_bytes(B, 512, M, N, K, mode), dtype=torch.uint8, device="cuda")
+                    fn = lambda i: cq.cq_gemm(cp[i % len(cp)], x, mode, ws, y)
+                    fn(0)
+                    t[mode] = time_graph(torch, stream, fn, len(cp))
+                paper.append({"N": N, "K": K, "B": B, "G": 512, "M": M, "ms_a16": round(t[0], 5), "ms_a8": round(t[1], 5),
+                              "a16_over_a8": round(t[0] / t[1], 3)})
+            del pw, cp
+            torch.cuda.empty_cache()
+    out["paper_h200_shapes_on_b200"] = paper
     out["decode_linears_w4g128"] = dec
     out["crossover"] = cross
     first = {}

@@ -25,8 +25,10 @@
  *   - Device layout: private, tiled and interleaved for 128-bit coalesced loads with the
  *     group parameters stored beside the codes of their tile; produced by cq_repack and
  *     inverted bit-exactly by cq_unpack.
- *   - Supported: B in 1..8; G in {32, 64, 128}; K % G == 0; M, N, K >= 1.  K and N need not be
- *     multiples of the 128 x 128 tile (the layout pads).
+ *   - Supported: B in 1..8; G in {32, 64, 128, 256, 512}; K % G == 0; M, N, K >= 1.  K and N need
+ *     not be multiples of the 128 x 128 tile (the layout pads).  For G = 256 / 512 the device layout
+ *     repeats a group's parameter record in each of its 128-wide tiles, so it is 8 (G/128 - 1) bytes
+ *     per group larger than the canonical format.
  */
 #ifndef CUBICQUANT_H_
 #define CUBICQUANT_H_
@@ -41,7 +43,7 @@ extern "C" {
 enum {
     CQ_OK = 0,
     CQ_ERR_INVALID_ARG = -1, /* null pointer, M/N/K <= 0, B outside 1..8, unknown mode */
-    CQ_ERR_UNSUPPORTED = -2, /* K % G != 0, G not in {32,64,128} */
+    CQ_ERR_UNSUPPORTED = -2, /* K % G != 0, G not in {32,64,128,256,512} */
     CQ_ERR_ALIGNMENT = -3,   /* a pointer is not 16-byte aligned */
     CQ_ERR_WORKSPACE = -4,   /* workspace_bytes smaller than cq_workspace_bytes() */
     CQ_ERR_ARCH = -5,        /* current device is not compute capability 10.x */

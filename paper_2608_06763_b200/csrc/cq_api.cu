@@ -39,7 +39,7 @@ Workspace plan_workspace(const Dims &d, int64_t M, int mode) {
 
 static int check_format(int B, int G, int64_t N, int64_t K) {
     if (B < 1 || B > 8 || N <= 0 || K <= 0 || G <= 0) return CQ_ERR_INVALID_ARG;
-    if (G != 32 && G != 64 && G != 128) return CQ_ERR_UNSUPPORTED;
+    if (G != 32 && G != 64 && G != 128 && G != 256 && G != 512) return CQ_ERR_UNSUPPORTED;
     if (K % G != 0) return CQ_ERR_UNSUPPORTED;
     return CQ_OK;
 }

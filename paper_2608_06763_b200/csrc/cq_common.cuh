@@ -5,7 +5,9 @@
 //
 //   The N x K code matrix is padded to Np x Kp (multiples of 128) and cut into 128 x 128 tiles,
 //   stored tile after tile with the K index fastest: tile (nb, kb) at (nb * KT + kb) * tile_bytes.
-//   A tile is   [codes: 8 row blocks of 16 rows x 128 k][params: 128 rows x (128/G) groups x 8 B].
+//   A tile is   [codes: 8 row blocks of 16 rows x 128 k][params: 128 rows x max(1, 128/G) records x 8 B];
+//   for G = 256 / 512 each 128-wide tile of a group repeats the group's record, so every tile stays
+//   self-contained (the layout is then larger than the canonical format by 8 (G/128 - 1) bytes per group).
 //   The 8-byte parameter record of a (row, group) is {float s, half a, half b}; the sign bit of s
 //   (s >= 0 in the format) flags a group that contains the reserved code pattern.
 //
@@ -36,7 +38,7 @@ struct Dims {
     int B, G;
     int64_t N, K;
     int NB, KT;       // tiles along N and K
-    int gpt;          // groups per tile = 128 / G
+    int gpt;          // parameter records per tile row = max(1, 128 / G)
     int code_bytes;   // bytes of the code part of a tile = 2048 * B
     int tile_bytes;   // code_bytes + 128 * gpt * 8
 };
@@ -46,7 +48,7 @@ __host__ __device__ inline Dims make_dims(int B, int G, int64_t N, int64_t K) {
     d.B = B; d.G = G; d.N = N; d.K = K;
     d.NB = (int)((N + TILE - 1) / TILE);
     d.KT = (int)((K + TILE - 1) / TILE);
-    d.gpt = TILE / G;
+    d.gpt = G >= TILE ? 1 : TILE / G;   // G = 256 / 512: every 128-wide tile of a group carries a copy of its record
     d.code_bytes = 2048 * B;
     d.tile_bytes = d.code_bytes + TILE * d.gpt * 8;
     return d;
@@ -115,7 +117,9 @@ __device__ inline unsigned fetch_u(const void *layout, const Dims &d, int64_t n,
 }
 
 __device__ inline GroupParams fetch_params(const void *layout, const Dims &d, int64_t n, int64_t kgroup) {
-    const int nb = (int)(n >> 7), kb = (int)(kgroup / d.gpt), gi = (int)(kgroup % d.gpt);
+    const int nb = (int)(n >> 7);
+    const int kb = d.G > TILE ? (int)(kgroup * (d.G / TILE)) : (int)(kgroup / d.gpt);   // first tile of a wide group
+    const int gi = d.G > TILE ? 0 : (int)(kgroup % d.gpt);
     const uint8_t *p = tile_ptr(layout, d, nb, kb) + d.code_bytes + (((int)(n & 127)) * d.gpt + gi) * 8;
     return *(const GroupParams *)p;
 }

@@ -84,7 +84,8 @@ __global__ void repack_params_kernel(const uint8_t *__restrict__ codes, const fl
     const int64_t tile = idx / per_tile;
     const int rem = (int)(idx % per_tile), r = rem / d.gpt, gi = rem % d.gpt;
     const int nb = (int)(tile / d.KT), kb = (int)(tile % d.KT);
-    const int64_t n = (int64_t)nb * TILE + r, kg = (int64_t)kb * d.gpt + gi, ng = d.K / d.G;
+    const int64_t n = (int64_t)nb * TILE + r, ng = d.K / d.G;
+    const int64_t kg = d.G > TILE ? ((int64_t)kb * TILE) / d.G : (int64_t)kb * d.gpt + gi;
     uint32_t sbits = 0;
     uint16_t ha = 0x3C00, hb = 0;  // (1, 0)
     if (n < d.N && kg < ng) {

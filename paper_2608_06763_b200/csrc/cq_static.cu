@@ -29,7 +29,7 @@ extern "C" int cq_gemv_static(const void *layout, int B, int G, const uint16_t *
                               int64_t K, void *stream) {
     using namespace cq;
     if (!layout || !x || !y || M <= 0 || N <= 0 || K <= 0 || B < 1 || B > 8) return CQ_ERR_INVALID_ARG;
-    if ((G != 32 && G != 64 && G != 128) || K % G != 0 || M > 16) return CQ_ERR_UNSUPPORTED;
+    if ((G != 32 && G != 64 && G != 128 && G != 256 && G != 512) || K % G != 0 || M > 16) return CQ_ERR_UNSUPPORTED;
     if (((uintptr_t)layout | (uintptr_t)x | (uintptr_t)y) & 15u) return CQ_ERR_ALIGNMENT;
     const Dims d = make_dims(B, G, N, K);
     const Workspace plan = plan_workspace(d, M, CQ_MODEL_DTYPE);

@@ -35,6 +35,8 @@ def test_sizes():
             assert cq.cq_effective_bits(B, G) == B + 64 / G
     assert cq.cq_layout_bytes(4, 128, 130, 128) == 2 * (128 * 128 // 2 + 128 * 8)  # N padded to 256
     assert cq.cq_layout_bytes(4, 48, 128, 96) == 0 and cq.cq_layout_bytes(4, 128, 128, 192) == 0
+    # G = 512: the record of a group is repeated in each of its four 128-wide tiles
+    assert cq.cq_layout_bytes(4, 512, 128, 1024) == 128 * 1024 // 2 + 8 * 128 * 8
     assert cq.cq_workspace_bytes(4, 128, 1, 4096, 4096, cq.CQ_MODEL_DTYPE) > 0
     assert cq.cq_workspace_bytes(4, 128, 1, 4096, 4096, cq.CQ_DYN_A8) > cq.cq_workspace_bytes(4, 128, 1, 4096, 4096, 0)
     assert cq.cq_workspace_bytes(4, 128, 1, 4096, 4096, 7) == 0
@@ -49,7 +51,7 @@ def test_argument_errors_are_found_before_any_launch():
     assert L.cq_gemm(one, 4, 128, one, one, 0, 128, 128, 0, one, 1 << 20, None) == -1
     assert L.cq_gemm(one, 4, 128, one, one, 1, 128, 128, 5, one, 1 << 20, None) == -1
     assert L.cq_gemm(one, 4, 128, one, one, 1, 128, 192, 0, one, 1 << 20, None) == -2   # K % G != 0
-    assert L.cq_gemm(one, 4, 256, one, one, 1, 128, 256, 0, one, 1 << 20, None) == -2   # G unsupported
+    assert L.cq_gemm(one, 4, 96, one, one, 1, 128, 192, 0, one, 1 << 20, None) == -2    # G unsupported
     assert L.cq_gemm(one, 4, 128, odd, one, 1, 128, 128, 0, one, 1 << 20, None) == -3
     assert L.cq_gemm(one, 4, 128, one, one, 1, 128, 128, 0, one, 16, None) == -4        # workspace too small
     assert L.cq_repack(None, one, one, one, 4, 128, 128, 128, one, None) == -1

@@ -25,10 +25,10 @@ def test_pack_codes_matches_oracle_bitstream(B):
     assert np.array_equal(got, oracle.pack(k, B))
 
 
-@pytest.mark.parametrize("G", [32, 64, 128])
+@pytest.mark.parametrize("G", [32, 64, 128, 256, 512])
 @pytest.mark.parametrize("B", ALL_B)
 def test_repack_unpack_roundtrip_bit_exact(B, G):
-    N, K = 200, 384  # N not a multiple of 128: padded rows
+    N, K = 200, 384 if G <= 128 else 1024  # N not a multiple of 128: padded rows
     c = logical_case(N, K, B, G, seed=30 + B)
     if B > 1:
         c.k[3, 5:9] = -(1 << (B - 1))
@@ -101,3 +101,24 @@ def test_a8_integer_partials_bit_exact(B):
     P = cq.cq_debug_a8_partials(c.pw, torch.from_numpy(rx8).cuda()).cpu().numpy()
     _, Pref = oracle.gemm_a8(c.codes, c.s, c.a, c.b, B, 64, c.K, rx8, rdx, want_partials=True)
     assert np.array_equal(P, Pref)
+
+
+@pytest.mark.parametrize("G", [256, 512])
+@pytest.mark.parametrize("B", [2, 5, 8])
+def test_wide_groups_levels_carriers_partials(B, G):
+    # group sizes of the paper's own kernel measurements
+    c = logical_case(72, 1024, B, G, seed=95 + B)
+    c.k[3, 300:310] = -(1 << (B - 1))
+    c = Case(c.k, c.s, c.a, c.b, B, G)
+    ref = oracle.levels_all(B, c.s, c.a, c.b)
+    got = cq.cq_decode_levels(c.pw).cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got - ref) <= 1e-6 * np.abs(ref))
+    assert np.array_equal(cq.cq_decode_carriers(c.pw).cpu().numpy(), oracle.carriers_all(B, c.a, c.b))
+    W = cq.cq_decode_weights(c.pw).cpu().numpy().astype(np.float64)
+    Wr = oracle.decode_dense(c.codes, c.s, c.a, c.b, B, G, c.K)
+    assert np.array_equal(np.sign(W), np.sign(Wr)) and np.all(np.abs(W - Wr) <= 1e-6 * np.abs(Wr))
+    x = datagen.activations(3, 1024, seed=96)
+    rx8, rdx = oracle.quantize_a8(x)
+    P = cq.cq_debug_a8_partials(c.pw, torch.from_numpy(rx8).cuda()).cpu().numpy()
+    _, Pref = oracle.gemm_a8(c.codes, c.s, c.a, c.b, B, G, c.K, rx8, rdx, want_partials=True)
+    assert np.array_equal(P, Pref) and np.abs(P).max() <= G * 127 * 127

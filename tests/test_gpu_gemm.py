@@ -138,3 +138,14 @@ def test_tensor_core_a8_gemm_all_widths_and_groups(B, G):
     x = datagen.activations(150, K, seed=181, outlier_cols=0.02)
     y, ref = run_both(c, x, cq.CQ_DYN_A8)
     check_y(y, ref, f"a8 tc B={B} G={G}")
+
+
+@pytest.mark.parametrize("mode", [cq.CQ_MODEL_DTYPE, cq.CQ_DYN_A8])
+@pytest.mark.parametrize("M", [1, 16, 64, 300])
+@pytest.mark.parametrize("B,G", [(2, 512), (5, 512), (8, 256), (4, 256)])
+def test_wide_groups_all_paths(B, G, M, mode):
+    # G = 256 / 512 (the group sizes of the paper's H200 measurements) through every kernel
+    c = encoded_case("normal", 200, 1024, B, G, seed=190 + B)
+    x = datagen.activations(M, 1024, seed=191, outlier_cols=0.01)
+    y, ref = run_both(c, x, mode)
+    check_y(y, ref, f"G={G} B={B} M={M} mode={mode}")
