@@ -26,7 +26,7 @@ Workspace plan_workspace(const Dims &d, int64_t M, int mode) {
     const int sk = (M > 16 && mode == CQ_MODEL_DTYPE) ? gemm_tc_split_k(d, M) : 1;
     const size_t n_ctr = (size_t)d.NB * (M > 16 ? (size_t)((M + bnt - 1) / bnt) : 1);
     w.counters_off = off; w.counters_bytes = align_up(n_ctr * 4, 256); off += w.counters_bytes;
-    size_t part = (size_t)d.NB * gp.max_slots * Mc * TILE * 4;
+    size_t part = (size_t)gp.ctas * 2 * Mc * TILE * 4;   // two partial slots per CTA
     if (sk > 1) { const size_t p2 = (size_t)sk * M * d.NB * TILE * 4; if (p2 > part) part = p2; }
     w.partial_off = off; w.partial_bytes = align_up(part, 256); off += w.partial_bytes;
     if (mode == CQ_DYN_A8) {

@@ -4,8 +4,8 @@
 // Work decomposition (balanced, persistent): the NB x KT grid of 128 x 128 weight tiles is cut
 // into P equal contiguous runs (P = resident CTAs of the whole GPU), one per CTA, in row-block
 // major order.  A run covers one or more row blocks; for each it streams its K range, and either
-// writes y (it covered the whole K range) or a partial sum into its slot; the last CTA to arrive
-// at a row block adds the slots in slot order (deterministic) and writes y.  The 8 warps of a CTA
+// writes y (it covered the whole K range) or a partial sum into one of its two slots; the CTA that completes
+// a row block adds the partials in K order (deterministic) and writes y.  The 8 warps of a CTA
 // own the 8 groups of 16 rows of a tile.
 //
 // Decode: a lane's 128-bit loads land directly in its MMA A-fragment positions (cq_common.cuh).
@@ -197,11 +197,14 @@ __device__ __forceinline__ void compute_tile(const TileRegs<B, TILE / G> &r, con
     });
 }
 
-// CTA index that owns linear tile `tile` when T tiles are cut into P runs [floor(c T / P), floor((c+1) T / P)).
-// Runs are cut on a "virtual" line in which every row block is KT tiles preceded by E overhead
-// units: a CTA whose run crosses into a new row block pays a second prologue and a second combine,
-// worth about E tiles, so it is given that many tiles fewer.  V = NB (KT + E) units are cut into P
-// runs [floor(c V / P), floor((c+1) V / P)); owner_of gives the CTA that holds tile (nb, kb).
+// How the NB x KT tiles are cut into one contiguous run per CTA.  Runs are cut on a "virtual" line
+// in which every row block is KT tiles preceded by E overhead units: a CTA whose run crosses into
+// a new row block pays a second prologue and a second combine, worth about E tiles, so it is given
+// that many tiles fewer.  With V units and P CTAs, CTA c owns the units [floor(V c / P), floor(V (c + 1) / P)).
+// (Giving the CTAs launched first on an SM longer runs, to offset the schedulers' preference for
+// the oldest warps, was measured and lost: the kernel is bound by issue slots, not by its tail.)
+__host__ __device__ inline int64_t cut_start(int64_t c, int64_t V, int64_t P) { return (V * c) / P; }
+// The CTA whose run holds tile (nb, kb): the largest c with floor(V c / P) <= v, i.e. V c < (v + 1) P.
 __host__ __device__ inline int owner_of(int nb, int kb, int KT, int E, int64_t V, int64_t P) {
     const int64_t v = (int64_t)nb * (KT + E) + E + kb;
     return (int)(((v + 1) * P - 1) / V);
@@ -212,7 +215,7 @@ __host__ __device__ inline int owner_of(int nb, int kb, int KT, int E, int64_t V
 template <int B, int G, int NT, int MODE>
 __global__ void __launch_bounds__(GEMV_THREADS, (NT == 1 && B <= 4 && G >= 64) ? CQ_GEMV_OCC_HI : 2)
 gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restrict__ x, const int8_t *__restrict__ xq,
-            int64_t x8_pitch, const float *__restrict__ dxs, uint16_t *__restrict__ y, int M, int max_slots, int E,
+            int64_t x8_pitch, const float *__restrict__ dxs, uint16_t *__restrict__ y, int M, int E,
             float *__restrict__ partial, int *__restrict__ counters) {
     constexpr int GPT = TILE / G;
     constexpr int L = B == 1 ? 1 : (1 << (B - 1));
@@ -227,7 +230,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int VT = d.KT + E;                       // virtual units per row block
     const int64_t V = (int64_t)d.NB * VT, P = gridDim.x;
-    const int64_t v_begin = ((int64_t)blockIdx.x * V) / P, v_end = ((int64_t)(blockIdx.x + 1) * V) / P;
+    const int64_t v_begin = cut_start(blockIdx.x, V, P), v_end = cut_start((int64_t)blockIdx.x + 1, V, P);
     if (threadIdx.x < 16) { s_max[threadIdx.x] = 0; s_inv[threadIdx.x] = 1.0f; }
     int8_t *ctab = nullptr;
     if constexpr (MODE == 1 && B >= 3) ctab = reinterpret_cast<int8_t *>(smem) + RT * (MAX_SUB * TILE + XS_PAD) + warp * 16 * L;
@@ -370,11 +373,10 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
 
         // ---- finish this row block
         const bool whole = (kb_begin == 0 && kb_end == d.KT);
-        const int c_first = owner_of(nb, 0, d.KT, E, V, P);
-        const int n_contrib = owner_of(nb, d.KT - 1, d.KT, E, V, P) - c_first + 1;
-        const int slot = (int)blockIdx.x - c_first;
+        // A run has at most two partial segments: one that starts inside a row block (its first) and
+        // one that starts a row block without finishing it (its last); each CTA owns two partial slots.
         const int64_t n_lo = (int64_t)nb * TILE + warp * 16 + g;
-        float *pslot = partial + ((size_t)nb * max_slots + slot) * (size_t)(M * TILE);
+        float *pslot = partial + ((size_t)blockIdx.x * 2 + (kb_begin > 0 ? 1 : 0)) * (size_t)(M * TILE);
 #pragma unroll
         for (int tb = 0; tb < NT; ++tb)
 #pragma unroll
@@ -390,26 +392,31 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                 }
             }
         if (!whole) {
-            // the last CTA to arrive at this row block adds the slots in slot order.  The barrier orders
-            // the CTA's partial stores before thread 0's release; its acquire plus the second barrier
-            // make the other CTAs' partials visible to every thread of the last one.
+            // The counter of a row block collects the tiles done; the CTA that completes it adds the
+            // partials in K order.  The barrier orders the CTA's partial stores before thread 0's release;
+            // its acquire plus the second barrier make the other CTAs' partials visible to every thread.
             __syncthreads();
             if (threadIdx.x == 0) {
                 int old;
-                asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(counters + nb) : "memory");
-                s_last = (old == n_contrib - 1);
+                asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(counters + nb), "r"(kb_end - kb_begin) : "memory");
+                s_last = (old + (kb_end - kb_begin) == d.KT);
             }
             __syncthreads();
             if (s_last) {
-                const float *pb = partial + (size_t)nb * max_slots * (size_t)(M * TILE);
+                const int c_first = owner_of(nb, 0, d.KT, E, V, P);   // its segment starts the row block: slot 0
+                const int n_contrib = owner_of(nb, d.KT - 1, d.KT, E, V, P) - c_first + 1;
+                const float *pb = partial + ((size_t)c_first * 2 + 1) * (size_t)(M * TILE);   // slot 1 of CTA c_first + q
                 for (int idx = threadIdx.x; idx < M * TILE; idx += GEMV_THREADS) {
                     const int m = idx / TILE, r = idx % TILE;
                     const int64_t n = (int64_t)nb * TILE + r;
                     float sum = 0.0f;
-                    for (int q0 = 0; q0 < n_contrib; q0 += 8) {  // eight independent loads in flight, added in slot order
+                    for (int q0 = 0; q0 < n_contrib; q0 += 8) {  // eight independent loads in flight, added in K order
                         float v[8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) v[i] = (q0 + i < n_contrib) ? __ldcg(pb + (size_t)(q0 + i) * (M * TILE) + idx) : 0.0f;
+                        for (int i = 0; i < 8; ++i) {
+                            const size_t off = (size_t)(q0 + i) * 2 * (M * TILE) - (q0 + i == 0 ? (size_t)(M * TILE) : 0);
+                            v[i] = (q0 + i < n_contrib) ? __ldcg(pb + off + idx) : 0.0f;
+                        }
 #pragma unroll
                         for (int i = 0; i < 8; ++i) sum += v[i];
                     }
@@ -423,12 +430,11 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
 
 template <int B, int G, int NT, int MODE>
 cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, const int8_t *xq, int64_t x8_pitch,
-                       const float *dxs, uint16_t *y, int M, int P, int max_slots, int E, float *partial, int *counters,
+                       const float *dxs, uint16_t *y, int M, int P, int max_run, int E, float *partial, int *counters,
                        cudaStream_t st) {
     constexpr int RT = 8 * NT;
     constexpr int L = B == 1 ? 1 : (1 << (B - 1));
-    const int64_t T = (int64_t)d.NB * d.KT;
-    int64_t sub64 = (T + P - 1) / P + 2;
+    int64_t sub64 = max_run;   // the longest run bounds the activation slice a CTA stages
     if (sub64 > d.KT) sub64 = d.KT;
     if (sub64 > MAX_SUB) sub64 = MAX_SUB;
     const int sub_tiles = (int)sub64;
@@ -454,29 +460,29 @@ cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, con
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = use_pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kern, (const uint8_t *)layout, d, x, xq, x8_pitch, dxs, y, M, max_slots, E, partial, counters);
+    return cudaLaunchKernelEx(&cfg, kern, (const uint8_t *)layout, d, x, xq, x8_pitch, dxs, y, M, E, partial, counters);
 }
 
 template <int B, int G>
 cudaError_t dispatch_nt_mode(const void *layout, const Dims &d, const uint16_t *x, const int8_t *xq, int64_t x8_pitch,
-                             const float *dxs, uint16_t *y, int M, int mode, int P, int max_slots, int E, float *partial,
+                             const float *dxs, uint16_t *y, int M, int mode, int P, int max_run, int E, float *partial,
                              int *counters, cudaStream_t st) {
     if (mode == 0) {
-        if (M <= 8) return launch_one<B, G, 1, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, E, partial, counters, st);
-        return launch_one<B, G, 2, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, E, partial, counters, st);
+        if (M <= 8) return launch_one<B, G, 1, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, st);
+        return launch_one<B, G, 2, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, st);
     }
-    if (M <= 8) return launch_one<B, G, 1, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, E, partial, counters, st);
-    return launch_one<B, G, 2, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_slots, E, partial, counters, st);
+    if (M <= 8) return launch_one<B, G, 1, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, st);
+    return launch_one<B, G, 2, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, st);
 }
 
 template <int B>
 cudaError_t dispatch_g(const void *layout, const Dims &d, const uint16_t *x, const int8_t *xq, int64_t x8_pitch,
-                       const float *dxs, uint16_t *y, int M, int mode, int P, int max_slots, int E, float *partial,
+                       const float *dxs, uint16_t *y, int M, int mode, int P, int max_run, int E, float *partial,
                        int *counters, cudaStream_t st) {
     switch (d.G) {
-        case 32: return dispatch_nt_mode<B, 32>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_slots, E, partial, counters, st);
-        case 64: return dispatch_nt_mode<B, 64>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_slots, E, partial, counters, st);
-        default: return dispatch_nt_mode<B, 128>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_slots, E, partial, counters, st);
+        case 32: return dispatch_nt_mode<B, 32>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_run, E, partial, counters, st);
+        case 64: return dispatch_nt_mode<B, 64>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_run, E, partial, counters, st);
+        default: return dispatch_nt_mode<B, 128>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_run, E, partial, counters, st);
     }
 }
 
@@ -492,14 +498,7 @@ GemvPlan gemv_plan(const Dims &d, int64_t M) {
     if (P > T) P = T;
     p.ctas = (int)P;
     p.overhead = (T / P >= 6) ? 3 : 0;   // a second prologue + combine costs about three tiles of work
-    const int E = p.overhead;
-    const int64_t V = (int64_t)d.NB * (d.KT + E);
-    int mx = 1;
-    for (int nb = 0; nb < d.NB; ++nb) {
-        const int c = owner_of(nb, d.KT - 1, d.KT, E, V, P) - owner_of(nb, 0, d.KT, E, V, P) + 1;
-        if (c > mx) mx = c;
-    }
-    p.max_slots = mx;
+    p.max_run = (int)(((int64_t)d.NB * (d.KT + p.overhead)) / P + 1);   // units, an upper bound of the tiles in a run
     return p;
 }
 
@@ -515,7 +514,8 @@ cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, ui
         cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, st);
         if (e != cudaSuccess) return e;
     }
-    const int Mi = (int)M, P = gp.ctas, ms = gp.max_slots, E = gp.overhead;
+    const int Mi = (int)M, P = gp.ctas, ms = gp.max_run;
+    const int E = gp.overhead;
     switch (d.B) {
         case 1: return dispatch_g<1>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, st);
         case 2: return dispatch_g<2>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, st);

@@ -22,7 +22,7 @@ cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *
 // Workspace carving (all offsets 256-byte aligned).
 struct Workspace {
     size_t counters_off, counters_bytes;   // int32 arrival counters, one per 128-row block
-    size_t partial_off, partial_bytes;     // fp32 split-K partial sums [NB][max_slots][M][128]
+    size_t partial_off, partial_bytes;     // fp32 split-K partial sums: small M [CTA][2][M][128]; GEMM [slice][M][Np]
     size_t x8_off, x8_bytes;               // Dynamic A8: int8 activation carrier [M][Kp]
     size_t dx_off, dx_bytes;               // Dynamic A8: row scales [M]
     size_t status_off;                     // int32 device status word (bounded waits report here)
@@ -32,7 +32,7 @@ Workspace plan_workspace(const Dims &d, int64_t M, int mode);
 
 // Decomposition of the small-M path: number of CTAs (one contiguous run of tiles each) and the
 // largest number of CTAs that contribute to one 128-row block.
-struct GemvPlan { int ctas, max_slots, overhead; };
+struct GemvPlan { int ctas, max_run, overhead; };
 GemvPlan gemv_plan(const Dims &d, int64_t M);
 
 // Small-M (M <= 16) split-K tensor-core GEMV, both activation modes.

@@ -30,5 +30,5 @@ def test_static_scratch_entry_rejects_what_does_not_fit():
     L = cq.lib()
     one = 16
     assert L.cq_gemv_static(one, 4, 128, one, one, 17, 128, 128, None) == -2          # more rows than the small-M path takes
-    assert L.cq_gemv_static(one, 4, 128, one, one, 16, 1 << 22, 1 << 15, None) == -4  # needs more than the built-in scratch
+    assert L.cq_gemv_static(one, 4, 128, one, one, 16, 1 << 29, 128, None) == -4      # its arrival counters alone exceed the built-in scratch
     assert L.cq_gemv_static(None, 4, 128, one, one, 1, 128, 128, None) == -1
