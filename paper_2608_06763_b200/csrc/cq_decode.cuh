@@ -74,19 +74,28 @@ __device__ __forceinline__ __half2 pair_T(const uint32_t (&w)[2 * B]) {
 struct RowCoef { __half2 a2, b2, c2; float s; };
 
 // Coefficients of q as a polynomial in T = k / 2^(B-1):  t = |T| rho, rho = 2^(B-1) / M, so
-// q = |T| (a rho + |T| (b rho^2 + |T| c rho^3)).
+// q = |T| (a rho + |T| (b rho^2 + |T| c rho^3)), c = 1 - a - b.  Built in half2 arithmetic from the
+// stored fp16 a and b (each coefficient is rounded to fp16 anyway; c rho^3 takes two FMA roundings).
+constexpr uint32_t half_bits_of(float v) {   // fp16 bit pattern of a positive normal v (round to nearest, ties up)
+    int e = 0;
+    float m = v;
+    while (m >= 2.0f) { m *= 0.5f; ++e; }
+    while (m < 1.0f) { m *= 2.0f; --e; }
+    const uint32_t frac = (uint32_t)((m - 1.0f) * 1024.0f + 0.5f);
+    return (uint32_t)((e + 15) << 10) + frac;   // a carry out of the fraction bumps the exponent
+}
 template <int B>
 __device__ __forceinline__ RowCoef make_coef(uint2 p) {
     RowCoef c;
     c.s = __uint_as_float(p.x & 0x7FFFFFFFu);
     if constexpr (B >= 3) {
         constexpr float rho = (float)(1 << (B - 1)) / (float)((1 << (B - 1)) - 1);
-        constexpr float rho2 = rho * rho, rho3 = rho * rho * rho;
-        const __half2 ab = as_h2(p.y);
-        const float a = __low2float(ab), b = __high2float(ab), cc = (1.0f - a) - b;
-        c.a2 = __float2half2_rn(a * rho);
-        c.b2 = __float2half2_rn(b * rho2);
-        c.c2 = __float2half2_rn(cc * rho3);
+        constexpr uint32_t r1 = h2dup(half_bits_of(rho)), r2 = h2dup(half_bits_of(rho * rho)), r3 = h2dup(half_bits_of(rho * rho * rho));
+        const __half2 a2 = as_h2(__byte_perm(p.y, 0, 0x1010)), b2 = as_h2(__byte_perm(p.y, 0, 0x3232));
+        c.a2 = __hmul2(a2, as_h2(r1));
+        c.b2 = __hmul2(b2, as_h2(r2));
+        const __half2 nr3 = as_h2(r3 | 0x80008000u);
+        c.c2 = __hfma2(b2, nr3, __hfma2(a2, nr3, as_h2(r3)));   // rho^3 - rho^3 a - rho^3 b
     }
     return c;
 }

@@ -47,6 +47,20 @@ __device__ __forceinline__ void mma_s8(int (&d)[4], const uint32_t (&a)[4], uint
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// the same MMAs with a zero C operand (the first MMA of a group: no accumulator registers to clear)
+__device__ __forceinline__ void mma_f16_z(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};\n"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.0f));
+}
+__device__ __forceinline__ void mma_s8_z(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm(
+        "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};\n"
+        : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "r"(0));
+}
+
 __device__ __forceinline__ uint4 ld_stream16(const void *p) {
     uint4 v;
     asm("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
@@ -91,14 +105,8 @@ __device__ __forceinline__ void group_model(const TileRegs<B, TILE / G> &r, cons
     const RowCoef c_lo = make_coef<B>(r.prm[0][GI]), c_hi = make_coef<B>(r.prm[1][GI]);
     // two accumulator sets so consecutive MMAs do not wait on each other
     float D[2][NT][4];
-#pragma unroll
-    for (int h = 0; h < 2; ++h)
-#pragma unroll
-        for (int tb = 0; tb < NT; ++tb)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) D[h][tb][i] = 0.0f;
     static_for<CPG>([&](auto jc) {
-        constexpr int j = GI * CPG + decltype(jc)::value;
+        constexpr int jj = decltype(jc)::value, j = GI * CPG + jj;
         uint32_t A[4];
         A[0] = level_pair<B, FIX>(pair_T<B, 4 * j + 0>(r.w), c_lo);
         A[1] = level_pair<B, FIX>(pair_T<B, 4 * j + 1>(r.w), c_hi);
@@ -107,7 +115,8 @@ __device__ __forceinline__ void group_model(const TileRegs<B, TILE / G> &r, cons
 #pragma unroll
         for (int tb = 0; tb < NT; ++tb) {
             const uint2 bf = *(const uint2 *)(xl + tb * 8 * XS + 16 * j);
-            mma_f16(D[j & 1][tb], A, bf.x, bf.y);
+            if constexpr (jj < 2) mma_f16_z(D[j & 1][tb], A, bf.x, bf.y);
+            else mma_f16(D[j & 1][tb], A, bf.x, bf.y);
         }
     });
 #pragma unroll
@@ -138,12 +147,8 @@ __device__ __forceinline__ void group_a8(const TileRegs<B, TILE / G> &r, const i
         __syncwarp();
     }
     int D[NT][4];
-#pragma unroll
-    for (int tb = 0; tb < NT; ++tb)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) D[tb][i] = 0;
     static_for<CPG / 2>([&](auto jc) {
-        constexpr int j = GI * CPG + 2 * decltype(jc)::value;
+        constexpr int jj = decltype(jc)::value, j = GI * CPG + 2 * jj;
         uint32_t A[4];
         // a0: row g chunk j; a1: row g+8 chunk j; a2: row g chunk j+1; a3: row g+8 chunk j+1
         static_for<4>([&](auto rc) {
@@ -168,7 +173,8 @@ __device__ __forceinline__ void group_a8(const TileRegs<B, TILE / G> &r, const i
         for (int tb = 0; tb < NT; ++tb) {
             const uint32_t b0 = *(const uint32_t *)(xl + tb * 8 * XS + 16 * j);
             const uint32_t b1 = *(const uint32_t *)(xl + tb * 8 * XS + 16 * (j + 1));
-            mma_s8(D[tb], A, b0, b1);
+            if constexpr (jj == 0) mma_s8_z(D[tb], A, b0, b1);
+            else mma_s8(D[tb], A, b0, b1);
         }
     });
     const float s_lo = __uint_as_float(p_lo.x & 0x7FFFFFFFu), s_hi = __uint_as_float(p_hi.x & 0x7FFFFFFFu);
