@@ -20,10 +20,16 @@
 //
 //   Stored code u = k + 2^(B-1) (offset binary; u = 0 is the reserved pattern), W1: u = bit.
 //   u is split into bit planes of power-of-two width (B = 3 -> 2+1, 5 -> 4+1, 6 -> 4+2,
-//   7 -> 4+2+1) so every field is extracted with shifts and masks only.  A plane of width pw puts
-//   pair p in word p / (16/pw) at bit (p % (16/pw)) * pw.  A lane's 2B words are stored as
-//   16-byte quads, quad Q of lane l at ((Q * 32) + l) * 16 inside the row block (then an 8-byte
-//   tail when 2B is not a multiple of 4), so every warp load is one contiguous 512- or 256-byte run.
+//   7 -> 4+2+1) so every field is extracted with shifts and masks only.  A plane of width pw holds
+//   16/pw pairs per word; pair_word / pair_pos below give the word and bit position of a pair.
+//   Write p = 4 j + 2 h + r (chunk j = 2 w + a, k half h, row half r) and n = 2 a + h:
+//     pw = 4: word 2 w + r, nibble n           -- a 16-bit half holds four codes of ONE row from one
+//     pw = 2: word w, field 2 n + r               32-wide k block, 4 bits apart, so it serves directly as
+//     pw = 1: word w / 2, bit 4 n + rho(w, r)     the selector of a byte-permute table lookup (Dynamic A8)
+//     pw = 8: word p / 2, byte p % 2
+//   A lane's 2B words are stored as 16-byte quads, quad Q of lane l at ((Q * 32) + l) * 16 inside
+//   the row block (then an 8-byte tail when 2B is not a multiple of 4), so every warp load is one
+//   contiguous 512- or 256-byte run.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -67,6 +73,17 @@ __host__ __device__ constexpr int plane_word_base(int B, int i) {   // first wor
     return 2 * plane_bit_offset(B, i);
 }
 
+// Word (inside its plane) and bit position (in the low 16-bit half; the pair's second code sits
+// 16 bits higher) of logical pair p = 4 j + 2 h + r in a plane of width pw.
+__host__ __device__ constexpr int pair_word(int pw, int p) {
+    const int r = p & 1, w = p >> 3;
+    return pw == 4 ? 2 * w + r : pw == 2 ? w : pw == 1 ? (w >> 1) : (p >> 1);
+}
+__host__ __device__ constexpr int pair_pos(int pw, int p) {
+    const int r = p & 1, h = (p >> 1) & 1, a = (p >> 2) & 1, w = p >> 3, n = 2 * a + h;
+    return pw == 4 ? 4 * n : pw == 2 ? 2 * (2 * n + r) : pw == 1 ? 4 * n + ((2 + 2 * (w & 1) + r) & 3) : 8 * (p & 1);
+}
+
 // byte offset of word W (0 .. 2B-1) of lane `lane` inside a row block
 __host__ __device__ inline int word_byte_offset(int B, int W, int lane) {
     const int nfq = (2 * B) / 4;
@@ -107,9 +124,9 @@ __device__ inline unsigned fetch_u(const void *layout, const Dims &d, int64_t n,
     unsigned u = 0;
     const int np = plane_count(d.B);
     for (int i = 0; i < np; ++i) {
-        const int pw = plane_width(d.B, i), ppw = 16 / pw;
-        const int W = plane_word_base(d.B, i) + s.pair / ppw;
-        const int pos = (s.pair % ppw) * pw + 16 * s.half;
+        const int pw = plane_width(d.B, i);
+        const int W = plane_word_base(d.B, i) + pair_word(pw, s.pair);
+        const int pos = pair_pos(pw, s.pair) + 16 * s.half;
         const uint32_t w = *(const uint32_t *)(rbp + word_byte_offset(d.B, W, s.lane));
         u |= ((w >> pos) & ((1u << pw) - 1u)) << plane_bit_offset(d.B, i);
     }

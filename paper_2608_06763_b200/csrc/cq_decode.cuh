@@ -1,7 +1,7 @@
 // Code-pair extraction and the half2 level evaluation shared by the small-M and large-M kernels.
 //
 // A lane's record (cq_common.cuh) holds 32 pairs of stored codes; pair P sits in one 32-bit word per
-// bit plane with its first code in the low and its second in the high 16 bits.  pair_T turns a
+// bit plane (pair_word / pair_pos) with its first code in the low and its second in the high 16 bits.  pair_T turns a
 // pair into the normalised signed codes T = k / 2^(B-1) as half2 with one mask (the code lands in
 // the fp16 mantissa under exponent bits 0x6400, value 1024 + u 2^pos) and one exact FMA; level_pair
 // evaluates the group's cubic in Horner form (Eq. gpu-horner) on it.
@@ -36,8 +36,8 @@ __device__ __forceinline__ uint32_t pair_codes(const uint32_t (&w)[2 * B]) {
     uint32_t u2 = 0;
     static_for<plane_count(B)>([&](auto ic) {
         constexpr int i = decltype(ic)::value;
-        constexpr int pw = plane_width(B, i), ppw = 16 / pw;
-        constexpr int W = plane_word_base(B, i) + P / ppw, pos = (P % ppw) * pw;
+        constexpr int pw = plane_width(B, i);
+        constexpr int W = plane_word_base(B, i) + pair_word(pw, P), pos = pair_pos(pw, P);
         constexpr uint32_t m = ((1u << pw) - 1u) * 0x00010001u;
         u2 |= ((w[W] >> pos) & m) << plane_bit_offset(B, i);
     });
@@ -50,7 +50,7 @@ __device__ __forceinline__ uint32_t pair_codes(const uint32_t (&w)[2 * B]) {
 template <int B, int P>
 __device__ __forceinline__ __half2 pair_T(const uint32_t (&w)[2 * B]) {
     if constexpr (plane_count(B) == 1) {
-        constexpr int PPW = 16 / B, W = P / PPW, pos0 = (P % PPW) * B;
+        constexpr int W = pair_word(B, P), pos0 = pair_pos(B, P);
         // B = 1 keeps the field off mantissa bit 0 (the offset constant must stay representable);
         // other widths shift by 8 when the field would leave the 10 mantissa bits
         constexpr int shl = (B == 1 && pos0 <= 6) ? 1 : 0;

@@ -55,11 +55,11 @@ __global__ void repack_codes_kernel(const uint8_t *__restrict__ codes, Dims d, i
     // which plane does word W belong to
     int pl = 0;
     for (int i = plane_count(d.B) - 1; i > 0; --i) if (W >= plane_word_base(d.B, i)) { pl = i; break; }
-    const int pw = plane_width(d.B, pl), ppw = 16 / pw, bo = plane_bit_offset(d.B, pl);
+    const int pw = plane_width(d.B, pl), bo = plane_bit_offset(d.B, pl);
     const int wi = W - plane_word_base(d.B, pl);
     uint32_t word = 0;
-    for (int q = 0; q < ppw; ++q) {
-        const int pair = wi * ppw + q;
+    for (int pair = 0; pair < 32; ++pair) {
+        if (pair_word(pw, pair) != wi) continue;
         for (int half = 0; half < 2; ++half) {
             int r, kk;
             weight_of(rb, lane, pair, half, r, kk);
@@ -67,7 +67,7 @@ __global__ void repack_codes_kernel(const uint8_t *__restrict__ codes, Dims d, i
             unsigned u;
             if (n < d.N && k < d.K) u = stored_from_field(d.B, canonical_field(codes + n * row_bytes, k, d.B, row_bytes));
             else u = (d.B == 1) ? 1u : (1u << (d.B - 1));  // padding: code 0 (W1: +1), its scale is 0
-            word |= ((u >> bo) & ((1u << pw) - 1u)) << (q * pw + 16 * half);
+            word |= ((u >> bo) & ((1u << pw) - 1u)) << (pair_pos(pw, pair) + 16 * half);
         }
     }
     uint8_t *dst = layout + (size_t)tile * d.tile_bytes + rb * 256 * d.B + word_byte_offset(d.B, W, lane);
