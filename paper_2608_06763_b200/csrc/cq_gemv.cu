@@ -28,7 +28,8 @@ namespace cq {
 namespace {
 
 constexpr int GEMV_THREADS = 256;
-constexpr int XS_PAD = 16;     // elements of padding per staged activation row (bank spread)
+constexpr int XS_PAD = 16;     // elements of padding per staged fp16 activation row (bank spread: 32 bytes)
+constexpr int XS_PAD8 = 32;    // the same for an INT8 row
 constexpr int MAX_SUB = 16;    // K tiles staged at a time (bounds shared memory)
 #ifndef CQ_GEMV_OCC_HI
 #define CQ_GEMV_OCC_HI 3       // resident CTAs per SM asked of the compiler for the light variants
@@ -128,53 +129,108 @@ __device__ __forceinline__ void group_model(const TileRegs<B, TILE / G> &r, cons
     }
 }
 
-// One group of a tile, Dynamic A8: carriers from the warp's table, INT8 MMAs, acc += s * P_g.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// Dynamic A8 operand order.  One INT8 MMA (k = 32) takes the 32-wide k block m of a tile.  Inside it
+// k = 16 a + 4 t + 2 h + e is held by lane t at byte n = 2 a + h of A register a0 / a1 (rows g / g+8)
+// for e = 0 and a2 / a3 for e = 1, which is where the layout's half-words put it.  The staged
+// activations use the same order: byte 32 m + 8 t + 4 e + n of a token row.
+//
+// Carriers (Eq. carrier) come from a per-(row, group) table indexed by the stored code u, so the
+// sign and the reserved pattern (u = 0 -> 0) are part of the table:
+//   B = 4: the table's two 8-byte halves (u < 8, u >= 8) live in registers; a half-word of four
+//          codes, masked to 3 bits each, is the selector of a byte permute into each half, and the
+//          codes' top bits (expanded to byte masks by two sign-replicating permutes) pick between them;
+//   B = 3: one 8-byte table, the selector assembled from the 2-bit and the 1-bit plane;
+//   B <= 2: the carriers are 0 / +-127, a constant table;
+//   B >= 5: the table stays in shared memory and is read per code.
+template <int B, int RR, int MI>
+__device__ __forceinline__ void a8_row_regs(const uint32_t (&w)[2 * B], const uint4 &tab, const int8_t *trow,
+                                            uint32_t &lo, uint32_t &hi) {
+    if constexpr (B == 4) {
+        const uint32_t word = w[2 * MI + RR];
+        const uint32_t ws = word & 0x77777777u, wh = ws >> 16, w4 = word << 4;
+        const uint32_t m_lo = prmt(w4, word, 0xD9C8u), m_hi = prmt(w4, word, 0xFBEAu);   // 0xFF where u >= 8
+        const uint32_t n_lo = prmt(tab.x, tab.y, ws), p_lo = prmt(tab.z, tab.w, ws);
+        const uint32_t n_hi = prmt(tab.x, tab.y, wh), p_hi = prmt(tab.z, tab.w, wh);
+        lo = (p_lo & m_lo) | (n_lo & ~m_lo);
+        hi = (p_hi & m_hi) | (n_hi & ~m_hi);
+    } else if constexpr (B == 3) {
+        constexpr int rho = (2 + 2 * (MI & 1) + RR) & 3;   // where the 1-bit plane keeps this selector's bits
+        const uint32_t x0 = RR ? (w[MI] >> 2) : w[MI];
+        const uint32_t w1 = w[4 + (MI >> 1)];
+        const uint32_t y = rho == 2 ? w1 : rho == 3 ? (w1 >> 1) : rho == 0 ? (w1 << 2) : (w1 << 1);
+        const uint32_t sel = (x0 & 0x33333333u) | (y & 0x44444444u);
+        lo = prmt(tab.x, tab.y, sel);
+        hi = prmt(tab.x, tab.y, sel >> 16);
+    } else if constexpr (B == 2) {
+        const uint32_t sel = (RR ? (w[MI] >> 2) : w[MI]) & 0x33333333u;
+        lo = prmt(0x7F008100u, 0u, sel);          // u = 0 reserved -> 0, 1 -> -127, 2 -> 0, 3 -> +127
+        hi = prmt(0x7F008100u, 0u, sel >> 16);
+    } else if constexpr (B == 1) {
+        constexpr int rho = (2 + 2 * (MI & 1) + RR) & 3;
+        const uint32_t sel = (w[MI >> 1] >> rho) & 0x11111111u;
+        lo = prmt(0x00007F81u, 0u, sel);          // bit 0 -> -127, bit 1 -> +127
+        hi = prmt(0x00007F81u, 0u, sel >> 16);
+    } else {
+        lo = 0; hi = 0;
+        static_for<4>([&](auto nc) {
+            constexpr int n = decltype(nc)::value, p = 4 * (2 * MI + (n >> 1)) + 2 * (n & 1) + RR;
+            const uint32_t u2 = pair_codes<B, p>(w);
+            lo |= (uint32_t)(uint8_t)trow[u2 & 0xFFFFu] << (8 * n);
+            hi |= (uint32_t)(uint8_t)trow[u2 >> 16] << (8 * n);
+        });
+    }
+}
+
+// One group of a tile, Dynamic A8: INT8 MMAs into int32 partials P_g, then acc += s * P_g.
+// xl = this lane's operand base (row g of the staged block, byte 8 t); ctab = this warp's table space.
 template <int B, int G, int NT, int GI>
 __device__ __forceinline__ void group_a8(const TileRegs<B, TILE / G> &r, const int8_t *xl, int XS, int8_t *ctab, int g,
                                          int t, float (&acc)[NT][4]) {
-    constexpr int CPG = G / 16;
+    constexpr int MPG = G / 32;                  // MMAs per group
     constexpr int L = B == 1 ? 1 : (1 << (B - 1));
+    constexpr int NE = 1 << B;                   // table entries per row
     const uint2 p_lo = r.prm[0][GI], p_hi = r.prm[1][GI];
-    if constexpr (B >= 3) {  // lane (g, t) fills entries i = t mod 4 of rows g and g + 8
+    uint4 tab_lo = make_uint4(0, 0, 0, 0), tab_hi = make_uint4(0, 0, 0, 0);
+    const int8_t *trow_lo = ctab + g * NE, *trow_hi = ctab + (g + 8) * NE;
+    if constexpr (B >= 3) {  // lane (g, t) fills magnitudes i = t mod 4 of rows g and g + 8: u = L + i and u = L - i
         __syncwarp();
         const __half2 ab_lo = as_h2(p_lo.y), ab_hi = as_h2(p_hi.y);
         const float a_lo = __low2float(ab_lo), b_lo = __high2float(ab_lo);
         const float a_hi = __low2float(ab_hi), b_hi = __high2float(ab_hi);
         for (int i = t; i < L; i += 4) {
-            ctab[g * L + i] = (int8_t)carrier_of(B, i, a_lo, b_lo);
-            ctab[(g + 8) * L + i] = (int8_t)carrier_of(B, i, a_hi, b_hi);
+            const int c_lo = carrier_of(B, i, a_lo, b_lo), c_hi = carrier_of(B, i, a_hi, b_hi);
+            ctab[g * NE + L + i] = (int8_t)c_lo;
+            ctab[g * NE + L - i] = (int8_t)(-c_lo);
+            ctab[(g + 8) * NE + L + i] = (int8_t)c_hi;
+            ctab[(g + 8) * NE + L - i] = (int8_t)(-c_hi);
         }
+        if (t == 0) { ctab[g * NE] = 0; ctab[(g + 8) * NE] = 0; }   // the reserved pattern
         __syncwarp();
+        if constexpr (B == 4) {
+            tab_lo = *reinterpret_cast<const uint4 *>(trow_lo);
+            tab_hi = *reinterpret_cast<const uint4 *>(trow_hi);
+        } else if constexpr (B == 3) {
+            const uint2 v0 = *reinterpret_cast<const uint2 *>(trow_lo), v1 = *reinterpret_cast<const uint2 *>(trow_hi);
+            tab_lo.x = v0.x; tab_lo.y = v0.y; tab_hi.x = v1.x; tab_hi.y = v1.y;
+        }
     }
     int D[NT][4];
-    static_for<CPG / 2>([&](auto jc) {
-        constexpr int jj = decltype(jc)::value, j = GI * CPG + 2 * jj;
+    static_for<MPG>([&](auto mc) {
+        constexpr int mi = decltype(mc)::value, MI = GI * MPG + mi;
         uint32_t A[4];
-        // a0: row g chunk j; a1: row g+8 chunk j; a2: row g chunk j+1; a3: row g+8 chunk j+1
-        static_for<4>([&](auto rc) {
-            constexpr int rr = decltype(rc)::value, jcx = j + (rr >> 1), hi_row = rr & 1;
-            uint32_t packed = 0;
-            static_for<2>([&](auto ec) {  // pairs (hi_row) and (2 + hi_row) hold k+0,1 and k+2,3
-                constexpr int e = decltype(ec)::value;
-                const uint32_t u2 = pair_codes<B, 4 * jcx + 2 * e + hi_row>(r.w);
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const unsigned u = (u2 >> (16 * hh)) & 0xFFFFu;
-                    const int code = signed_code(B, u);
-                    int rv;
-                    if constexpr (B <= 2) rv = 127 * code;
-                    else { rv = ctab[(g + 8 * hi_row) * L + abs(code)]; rv = code < 0 ? -rv : rv; }
-                    packed |= ((uint32_t)rv & 0xFFu) << (8 * (2 * e + hh));
-                }
-            });
-            A[rr] = packed;
-        });
+        a8_row_regs<B, 0, MI>(r.w, tab_lo, trow_lo, A[0], A[2]);
+        a8_row_regs<B, 1, MI>(r.w, tab_hi, trow_hi, A[1], A[3]);
 #pragma unroll
         for (int tb = 0; tb < NT; ++tb) {
-            const uint32_t b0 = *(const uint32_t *)(xl + tb * 8 * XS + 16 * j);
-            const uint32_t b1 = *(const uint32_t *)(xl + tb * 8 * XS + 16 * (j + 1));
-            if constexpr (jj == 0) mma_s8_z(D[tb], A, b0, b1);
-            else mma_s8(D[tb], A, b0, b1);
+            const uint2 bf = *reinterpret_cast<const uint2 *>(xl + tb * 8 * XS + 32 * MI);
+            if constexpr (mi == 0) mma_s8_z(D[tb], A, bf.x, bf.y);
+            else mma_s8(D[tb], A, bf.x, bf.y);
         }
     });
     const float s_lo = __uint_as_float(p_lo.x & 0x7FFFFFFFu), s_hi = __uint_as_float(p_hi.x & 0x7FFFFFFFu);
@@ -228,6 +284,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
     constexpr int RT = 8 * NT;       // staged token rows (rows >= M are zero)
     constexpr int NBUF = (B <= 4) ? 3 : 2;
     constexpr int ES = MODE == 0 ? 2 : 1;  // bytes per staged activation element
+    constexpr int XPAD = MODE == 0 ? XS_PAD : XS_PAD8;
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ float s_inv[16];
     __shared__ unsigned s_max[16];
@@ -239,7 +296,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
     const int64_t v_begin = cut_start(blockIdx.x, V, P), v_end = cut_start((int64_t)blockIdx.x + 1, V, P);
     if (threadIdx.x < 16) { s_max[threadIdx.x] = 0; s_inv[threadIdx.x] = 1.0f; }
     int8_t *ctab = nullptr;
-    if constexpr (MODE == 1 && B >= 3) ctab = reinterpret_cast<int8_t *>(smem) + RT * (MAX_SUB * TILE + XS_PAD) + warp * 16 * L;
+    if constexpr (MODE == 1 && B >= 3) ctab = reinterpret_cast<int8_t *>(smem) + RT * (MAX_SUB * TILE + XS_PAD8) + warp * 16 * (1 << B);
 
     bool first_slice = true;
     for (int64_t v = v_begin; v < v_end;) {
@@ -257,7 +314,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
 
         for (int ks = kb_begin; ks < kb_end; ks += MAX_SUB) {
             const int ke = min(kb_end, ks + MAX_SUB);
-            const int slice_k = (ke - ks) * TILE, XS = slice_k + XS_PAD;
+            const int slice_k = (ke - ks) * TILE, XS = slice_k + XPAD;
             const int64_t k_base = (int64_t)ks * TILE;
             const uint8_t *tile0 = layout + ((size_t)nb * d.KT + ks) * (size_t)d.tile_bytes;
             const uint8_t *wl = tile0 + warp * 256 * B + lane * 16;                     // next tile to load (codes)
@@ -344,6 +401,23 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                 }
             } else {
                 if (threadIdx.x < 16) s_inv[threadIdx.x] = threadIdx.x < M ? dxs[threadIdx.x] * (1.0f / 127.0f) : 0.0f;
+                // bring the carriers into MMA operand order (see a8_row_regs): the 16-byte chunks c and
+                // c ^ 1 (same warp) share one 32-byte block, so both are read before either is rewritten
+                for (int m = 0; m < M; ++m) {
+                    uint8_t *blk = smem + (size_t)m * XS + (size_t)(c >> 1) * 32 + 2 * (c & 1);
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (c < cpr) v = *(const uint4 *)(smem + (size_t)m * XS + (size_t)c * 16);
+                    __syncwarp();
+                    if (c < cpr) {
+                        const uint32_t ws[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {   // bytes k+0, k+2 (e = 0) | k+1, k+3 (e = 1)
+                            const uint32_t pr = prmt(ws[q], 0u, 0x3120u);
+                            *(uint16_t *)(blk + 8 * q) = (uint16_t)pr;
+                            *(uint16_t *)(blk + 8 * q + 4) = (uint16_t)(pr >> 16);
+                        }
+                    }
+                }
             }
             __syncthreads();
             if (MODE == 0 && threadIdx.x < 16) s_max[threadIdx.x] = 0;  // next slice's maxima start from zero
@@ -354,7 +428,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
             for (int tb = 0; tb < NT; ++tb)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) acc[tb][i] = 0.0f;
-            const uint8_t *xcur = smem + (size_t)(g * XS + 4 * t) * ES;  // this lane's B-fragment base, current tile
+            const uint8_t *xcur = smem + (size_t)(g * XS + (MODE == 0 ? 4 : 8) * t) * ES;  // this lane's B-fragment base, current tile
             int to_load = (ke - ks) - NBUF;                              // tiles not yet requested
             for (int left = ke - ks; left > 0; left -= NBUF) {
                 static_for<NBUF>([&](auto ic) {
@@ -445,7 +519,7 @@ cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, con
     if (sub64 > MAX_SUB) sub64 = MAX_SUB;
     const int sub_tiles = (int)sub64;
     const int XS = sub_tiles * TILE + XS_PAD;
-    size_t smem = MODE == 0 ? (size_t)RT * XS * 2 : (size_t)RT * (MAX_SUB * TILE + XS_PAD) + 8 * 16 * L;
+    size_t smem = MODE == 0 ? (size_t)RT * XS * 2 : (size_t)RT * (MAX_SUB * TILE + XS_PAD8) + (B >= 3 ? 8 * 16 * (1 << B) : 0);
     auto kern = gemv_kernel<B, G, NT, MODE>;
     static bool attr_done = false;
     if (smem > 48 * 1024 && !attr_done) {

@@ -201,7 +201,8 @@ __global__ void a8_partials_kernel(const void *__restrict__ layout, Dims d, cons
 // One block per row (Eq. a8-activation-scale, Eq. a8-activation-quantization).  fp32 arithmetic:
 // xbar = max(max|x|, 1e-10f); dx = xbar / 127 (IEEE); x8 = clip(round-half-away(x / dx), +-127).
 // Written with a row pitch so the GEMM can ask for a padded carrier.
-__global__ void __launch_bounds__(256) quantize_a8_kernel(const uint16_t *__restrict__ x, int64_t M, int64_t K,
+// plain version for rows whose length or addresses do not allow 16-byte accesses
+__global__ void __launch_bounds__(256) quantize_a8_scalar_kernel(const uint16_t *__restrict__ x, int64_t M, int64_t K,
                                                          int8_t *__restrict__ x8, int64_t x8_pitch,
                                                          float *__restrict__ dx) {
     __shared__ float red[8];
@@ -234,6 +235,63 @@ __global__ void __launch_bounds__(256) quantize_a8_kernel(const uint16_t *__rest
             q = (int)r;
         }
         orow[j] = (int8_t)q;
+    }
+}
+
+// 16-byte loads, 8-byte stores: K and the pitch multiples of 8, x 16-byte and x8 8-byte aligned
+__global__ void __launch_bounds__(1024) quantize_a8_kernel(const uint16_t *__restrict__ x, int64_t M, int64_t K,
+                                                          int8_t *__restrict__ x8, int64_t x8_pitch,
+                                                          float *__restrict__ dx) {
+    // the kernel launched next may start now (its first steps do not touch what this one writes)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    __shared__ unsigned red[32];
+    __shared__ float s_d;
+    const int64_t m = blockIdx.x;
+    const uint4 *row = reinterpret_cast<const uint4 *>(x + m * K);   // K % 8 == 0 and x is 16-byte aligned
+    const int64_t chunks = K >> 3;                                    // 8 values per 16-byte chunk
+    // pass 1: the row maximum of |x| as a bf16 bit pattern (for non-NaN values the integer order of
+    // the patterns with the sign cleared is the order of the magnitudes); the first chunk stays in registers
+    uint4 keep = make_uint4(0, 0, 0, 0);
+    unsigned mx = 0;
+    for (int64_t j = threadIdx.x; j < chunks; j += blockDim.x) {
+        const uint4 v = row[j];
+        if (j == threadIdx.x) keep = v;
+        const uint32_t ws[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { mx = max(mx, ws[q] & 0x7FFFu); mx = max(mx, (ws[q] >> 16) & 0x7FFFu); }
+    }
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        unsigned v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0u;
+        v = __reduce_max_sync(0xffffffffu, v);
+        if (threadIdx.x == 0) {
+            const float xbar = fmaxf(__uint_as_float(v << 16), 1e-10f);
+            const float d = __fdiv_rn(xbar, 127.0f);
+            s_d = d;
+            dx[m] = d;
+        }
+    }
+    __syncthreads();
+    const float d = s_d;
+    // pass 2: x8 = clip(round_half_away(x / d)), 8 values per thread and step
+    uint2 *orow = reinterpret_cast<uint2 *>(x8 + m * x8_pitch);
+    const int64_t out_chunks = x8_pitch >> 3;
+    for (int64_t j = threadIdx.x; j < out_chunks; j += blockDim.x) {
+        uint32_t out[2] = {0u, 0u};
+        if (j < chunks) {
+            const uint4 v = (j == threadIdx.x) ? keep : row[j];
+            const uint32_t ws[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const uint32_t bits = (q & 1) ? (ws[q >> 1] & 0xFFFF0000u) : (ws[q >> 1] << 16);
+                float r = roundf(__fdiv_rn(__uint_as_float(bits), d));  // halves away from zero
+                r = fminf(fmaxf(r, -127.0f), 127.0f);
+                out[q >> 2] |= ((uint32_t)(int)r & 0xFFu) << (8 * (q & 3));
+            }
+        }
+        orow[j] = make_uint2(out[0], out[1]);
     }
 }
 
@@ -288,7 +346,16 @@ cudaError_t launch_a8_partials(const void *layout, const Dims &d, const int8_t *
 }
 cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, int64_t x8_pitch, float *dx,
                                cudaStream_t st) {
-    quantize_a8_kernel<<<(unsigned)M, 256, 0, st>>>(x, M, K, x8, x8_pitch, dx);
+    const bool wide = K % 8 == 0 && x8_pitch % 8 == 0 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0 &&
+                      (reinterpret_cast<uintptr_t>(x8) & 7u) == 0;
+    if (!wide) {
+        quantize_a8_scalar_kernel<<<(unsigned)M, 256, 0, st>>>(x, M, K, x8, x8_pitch, dx);
+        return cudaGetLastError();
+    }
+    int64_t threads = ((K >> 3) + 31) / 32 * 32;   // one 8-value chunk per thread when the row is short enough
+    if (threads > 1024) threads = 1024;
+    if (M > 64 && threads > 256) threads = 256;    // many rows: smaller CTAs fill the SMs better
+    quantize_a8_kernel<<<(unsigned)M, (unsigned)threads, 0, st>>>(x, M, K, x8, x8_pitch, dx);
     return cudaGetLastError();
 }
 
