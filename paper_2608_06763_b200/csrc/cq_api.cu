@@ -182,7 +182,7 @@ int cq_gemm_host(const void *layout, int B, int G, const uint16_t *x_host, uint1
 
 int cq_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, float *dx, void *stream) {
     if (!x || !x8 || !dx || M <= 0 || K <= 0) return CQ_ERR_INVALID_ARG;
-    return wrap(launch_quantize_a8(x, M, K, x8, K, dx, (cudaStream_t)stream));
+    return wrap(launch_quantize_a8(x, M, K, x8, K, dx, false, (cudaStream_t)stream));
 }
 
 #define CQ_DEBUG_PROLOGUE()                                   \

@@ -213,23 +213,26 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
                                 __syncwarp();
                             }
                         }
-                        static_for<CPGH>([&](auto jc) {
-                            constexpr int j = 4 * JH + decltype(gc)::value * CPGH + decltype(jc)::value;
-                            auto carrier = [&](unsigned u, const int8_t *trow) -> uint32_t {
-                                if constexpr (B >= 3) return (uint32_t)(uint8_t)trow[u];
-                                else return (uint32_t)(uint8_t)(int8_t)(127 * signed_code(B, u));
-                            };
-                            const int8_t *t_lo = tab + g * NCODE, *t_hi = tab + (g + 8) * NCODE;
-                            const uint32_t u0 = pair_codes<B, 4 * j + 0>(w), u1 = pair_codes<B, 4 * j + 1>(w);
-                            const uint32_t u2 = pair_codes<B, 4 * j + 2>(w), u3 = pair_codes<B, 4 * j + 3>(w);
-                            const uint32_t lo = carrier(u0 & 0xFFFFu, t_lo) | (carrier(u0 >> 16, t_lo) << 8) |
-                                                (carrier(u2 & 0xFFFFu, t_lo) << 16) | (carrier(u2 >> 16, t_lo) << 24);
-                            const uint32_t hi = carrier(u1 & 0xFFFFu, t_hi) | (carrier(u1 >> 16, t_hi) << 8) |
-                                                (carrier(u3 & 0xFFFFu, t_hi) << 16) | (carrier(u3 >> 16, t_hi) << 24);
-                            // k offset inside the block: 16 j + 4 tq bytes -> 16-byte chunk j, swizzled by the row
-                            const int off = ((j ^ g) * 16) + tq * 4;
-                            *(uint32_t *)(row_lo + off) = lo;
-                            *(uint32_t *)(row_hi + off) = hi;
+                        // carriers of the group's 32-wide k blocks, straight into the MMA operand order
+                        // (a8_row_regs): lane tq holds bytes 8 tq .. 8 tq + 7 of block m for rows g and g + 8
+                        const int8_t *t_lo = tab + g * NCODE, *t_hi = tab + (g + 8) * NCODE;
+                        uint4 tab_lo = make_uint4(0, 0, 0, 0), tab_hi = make_uint4(0, 0, 0, 0);
+                        if constexpr (B == 4) {
+                            tab_lo = *reinterpret_cast<const uint4 *>(t_lo);
+                            tab_hi = *reinterpret_cast<const uint4 *>(t_hi);
+                        } else if constexpr (B == 3) {
+                            const uint2 v0 = *reinterpret_cast<const uint2 *>(t_lo), v1 = *reinterpret_cast<const uint2 *>(t_hi);
+                            tab_lo.x = v0.x; tab_lo.y = v0.y; tab_hi.x = v1.x; tab_hi.y = v1.y;
+                        }
+                        static_for<CPGH / 2>([&](auto mc) {
+                            constexpr int MI = 2 * JH + decltype(gc)::value * (CPGH / 2) + decltype(mc)::value;
+                            uint2 lo, hi;
+                            a8_row_regs<B, 0, MI>(w, tab_lo, t_lo, lo.x, lo.y);
+                            a8_row_regs<B, 1, MI>(w, tab_hi, t_hi, hi.x, hi.y);
+                            // bytes 32 MI + 8 tq of the row: 16-byte chunk 2 MI + tq / 2, swizzled by the row
+                            const int off = (((2 * MI + (tq >> 1)) ^ g) * 16) + (tq & 1) * 8;
+                            *(uint2 *)(row_lo + off) = lo;
+                            *(uint2 *)(row_hi + off) = hi;
                         });
                     });
                 };
@@ -337,7 +340,7 @@ cudaError_t launch_gemm_a8_tc(const void *layout, const Dims &d, const uint16_t 
     float *dxs = reinterpret_cast<float *>(ws + plan.dx_off);
     int *status = reinterpret_cast<int *>(ws + plan.status_off);
     const int64_t pitch = (int64_t)d.KT * TILE;
-    cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, st);
+    cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, true, st);
     if (e != cudaSuccess) return e;
     switch (d.B) {
         case 1: return launch_a8_b<1>(layout, d, xq, pitch, dxs, y, M, status, st);

@@ -129,64 +129,6 @@ __device__ __forceinline__ void group_model(const TileRegs<B, TILE / G> &r, cons
     }
 }
 
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-    return d;
-}
-
-// Dynamic A8 operand order.  One INT8 MMA (k = 32) takes the 32-wide k block m of a tile.  Inside it
-// k = 16 a + 4 t + 2 h + e is held by lane t at byte n = 2 a + h of A register a0 / a1 (rows g / g+8)
-// for e = 0 and a2 / a3 for e = 1, which is where the layout's half-words put it.  The staged
-// activations use the same order: byte 32 m + 8 t + 4 e + n of a token row.
-//
-// Carriers (Eq. carrier) come from a per-(row, group) table indexed by the stored code u, so the
-// sign and the reserved pattern (u = 0 -> 0) are part of the table:
-//   B = 4: the table's two 8-byte halves (u < 8, u >= 8) live in registers; a half-word of four
-//          codes, masked to 3 bits each, is the selector of a byte permute into each half, and the
-//          codes' top bits (expanded to byte masks by two sign-replicating permutes) pick between them;
-//   B = 3: one 8-byte table, the selector assembled from the 2-bit and the 1-bit plane;
-//   B <= 2: the carriers are 0 / +-127, a constant table;
-//   B >= 5: the table stays in shared memory and is read per code.
-template <int B, int RR, int MI>
-__device__ __forceinline__ void a8_row_regs(const uint32_t (&w)[2 * B], const uint4 &tab, const int8_t *trow,
-                                            uint32_t &lo, uint32_t &hi) {
-    if constexpr (B == 4) {
-        const uint32_t word = w[2 * MI + RR];
-        const uint32_t ws = word & 0x77777777u, wh = ws >> 16, w4 = word << 4;
-        const uint32_t m_lo = prmt(w4, word, 0xD9C8u), m_hi = prmt(w4, word, 0xFBEAu);   // 0xFF where u >= 8
-        const uint32_t n_lo = prmt(tab.x, tab.y, ws), p_lo = prmt(tab.z, tab.w, ws);
-        const uint32_t n_hi = prmt(tab.x, tab.y, wh), p_hi = prmt(tab.z, tab.w, wh);
-        lo = (p_lo & m_lo) | (n_lo & ~m_lo);
-        hi = (p_hi & m_hi) | (n_hi & ~m_hi);
-    } else if constexpr (B == 3) {
-        constexpr int rho = (2 + 2 * (MI & 1) + RR) & 3;   // where the 1-bit plane keeps this selector's bits
-        const uint32_t x0 = RR ? (w[MI] >> 2) : w[MI];
-        const uint32_t w1 = w[4 + (MI >> 1)];
-        const uint32_t y = rho == 2 ? w1 : rho == 3 ? (w1 >> 1) : rho == 0 ? (w1 << 2) : (w1 << 1);
-        const uint32_t sel = (x0 & 0x33333333u) | (y & 0x44444444u);
-        lo = prmt(tab.x, tab.y, sel);
-        hi = prmt(tab.x, tab.y, sel >> 16);
-    } else if constexpr (B == 2) {
-        const uint32_t sel = (RR ? (w[MI] >> 2) : w[MI]) & 0x33333333u;
-        lo = prmt(0x7F008100u, 0u, sel);          // u = 0 reserved -> 0, 1 -> -127, 2 -> 0, 3 -> +127
-        hi = prmt(0x7F008100u, 0u, sel >> 16);
-    } else if constexpr (B == 1) {
-        constexpr int rho = (2 + 2 * (MI & 1) + RR) & 3;
-        const uint32_t sel = (w[MI >> 1] >> rho) & 0x11111111u;
-        lo = prmt(0x00007F81u, 0u, sel);          // bit 0 -> -127, bit 1 -> +127
-        hi = prmt(0x00007F81u, 0u, sel >> 16);
-    } else {
-        lo = 0; hi = 0;
-        static_for<4>([&](auto nc) {
-            constexpr int n = decltype(nc)::value, p = 4 * (2 * MI + (n >> 1)) + 2 * (n & 1) + RR;
-            const uint32_t u2 = pair_codes<B, p>(w);
-            lo |= (uint32_t)(uint8_t)trow[u2 & 0xFFFFu] << (8 * n);
-            hi |= (uint32_t)(uint8_t)trow[u2 >> 16] << (8 * n);
-        });
-    }
-}
-
 // One group of a tile, Dynamic A8: INT8 MMAs into int32 partials P_g, then acc += s * P_g.
 // xl = this lane's operand base (row g of the staged block, byte 8 t); ctab = this warp's table space.
 template <int B, int G, int NT, int GI>
@@ -344,7 +286,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                             const int64_t k = k_base + (int64_t)c * 8;
                             if (k < d.K) src = x + (int64_t)m * d.K + k;   // K % 8 == 0 always
                         } else {
-                            src = xq + (int64_t)m * x8_pitch + k_base + c * 16;  // pitch multiple of 128, zero beyond K
+                            src = xq + (int64_t)m * x8_pitch + k_base + c * 16;  // already in MMA operand order; pitch multiple of 128, zero beyond K
                         }
                     }
                     if (src) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
@@ -401,23 +343,6 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                 }
             } else {
                 if (threadIdx.x < 16) s_inv[threadIdx.x] = threadIdx.x < M ? dxs[threadIdx.x] * (1.0f / 127.0f) : 0.0f;
-                // bring the carriers into MMA operand order (see a8_row_regs): the 16-byte chunks c and
-                // c ^ 1 (same warp) share one 32-byte block, so both are read before either is rewritten
-                for (int m = 0; m < M; ++m) {
-                    uint8_t *blk = smem + (size_t)m * XS + (size_t)(c >> 1) * 32 + 2 * (c & 1);
-                    uint4 v = make_uint4(0, 0, 0, 0);
-                    if (c < cpr) v = *(const uint4 *)(smem + (size_t)m * XS + (size_t)c * 16);
-                    __syncwarp();
-                    if (c < cpr) {
-                        const uint32_t ws[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {   // bytes k+0, k+2 (e = 0) | k+1, k+3 (e = 1)
-                            const uint32_t pr = prmt(ws[q], 0u, 0x3120u);
-                            *(uint16_t *)(blk + 8 * q) = (uint16_t)pr;
-                            *(uint16_t *)(blk + 8 * q + 4) = (uint16_t)(pr >> 16);
-                        }
-                    }
-                }
             }
             __syncthreads();
             if (MODE == 0 && threadIdx.x < 16) s_max[threadIdx.x] = 0;  // next slice's maxima start from zero
@@ -591,7 +516,7 @@ cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, ui
     float *dxs = reinterpret_cast<float *>(ws + plan.dx_off);
     const int64_t pitch = (int64_t)d.KT * TILE;
     if (mode == 1) {
-        cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, st);
+        cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, true, st);
         if (e != cudaSuccess) return e;
     }
     const int Mi = (int)M, P = gp.ctas, ms = gp.max_run;

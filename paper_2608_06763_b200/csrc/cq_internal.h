@@ -17,7 +17,7 @@ cudaError_t launch_decode_carriers(const void *layout, const Dims &d, int8_t *ca
 cudaError_t launch_decode_weights(const void *layout, const Dims &d, float *What, cudaStream_t st);
 cudaError_t launch_a8_partials(const void *layout, const Dims &d, const int8_t *x8, int64_t M, int32_t *P, cudaStream_t st);
 cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, int64_t x8_pitch, float *dx,
-                               cudaStream_t st);
+                               bool operand_order, cudaStream_t st);
 
 // Workspace carving (all offsets 256-byte aligned).
 struct Workspace {

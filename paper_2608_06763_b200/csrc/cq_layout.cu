@@ -239,6 +239,7 @@ __global__ void __launch_bounds__(256) quantize_a8_scalar_kernel(const uint16_t 
 }
 
 // 16-byte loads, 8-byte stores: K and the pitch multiples of 8, x 16-byte and x8 8-byte aligned
+template <bool OPERAND_ORDER>
 __global__ void __launch_bounds__(1024) quantize_a8_kernel(const uint16_t *__restrict__ x, int64_t M, int64_t K,
                                                           int8_t *__restrict__ x8, int64_t x8_pitch,
                                                           float *__restrict__ dx) {
@@ -291,7 +292,19 @@ __global__ void __launch_bounds__(1024) quantize_a8_kernel(const uint16_t *__res
                 out[q >> 2] |= ((uint32_t)(int)r & 0xFFu) << (8 * (q & 3));
             }
         }
-        orow[j] = make_uint2(out[0], out[1]);
+        if constexpr (!OPERAND_ORDER) {
+            orow[j] = make_uint2(out[0], out[1]);
+        } else {
+            // k = 32 m + 16 a + 4 t + 2 h + e goes to byte 32 m + 8 t + 4 e + 2 a + h (cq_decode.cuh); this
+            // chunk holds t = 2 (j & 1) + {0, 1} of half a = (j >> 1) & 1
+            uint8_t *blk = reinterpret_cast<uint8_t *>(x8 + m * x8_pitch) + (j >> 2) * 32 + 2 * ((j >> 1) & 1) + 16 * (j & 1);
+#pragma unroll
+            for (int tt = 0; tt < 2; ++tt) {
+                const uint32_t pr = __byte_perm(out[tt], 0u, 0x3120);   // bytes (k+0, k+2 | k+1, k+3)
+                *reinterpret_cast<uint16_t *>(blk + 8 * tt) = (uint16_t)pr;
+                *reinterpret_cast<uint16_t *>(blk + 8 * tt + 4) = (uint16_t)(pr >> 16);
+            }
+        }
     }
 }
 
@@ -345,9 +358,10 @@ cudaError_t launch_a8_partials(const void *layout, const Dims &d, const int8_t *
     return cudaGetLastError();
 }
 cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, int64_t x8_pitch, float *dx,
-                               cudaStream_t st) {
+                               bool operand_order, cudaStream_t st) {
     const bool wide = K % 8 == 0 && x8_pitch % 8 == 0 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0 &&
                       (reinterpret_cast<uintptr_t>(x8) & 7u) == 0;
+    if (operand_order && !(wide && x8_pitch % 32 == 0)) return cudaErrorInvalidValue;   // internal callers pad the pitch to 128
     if (!wide) {
         quantize_a8_scalar_kernel<<<(unsigned)M, 256, 0, st>>>(x, M, K, x8, x8_pitch, dx);
         return cudaGetLastError();
@@ -355,7 +369,8 @@ cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *
     int64_t threads = ((K >> 3) + 31) / 32 * 32;   // one 8-value chunk per thread when the row is short enough
     if (threads > 1024) threads = 1024;
     if (M > 64 && threads > 256) threads = 256;    // many rows: smaller CTAs fill the SMs better
-    quantize_a8_kernel<<<(unsigned)M, (unsigned)threads, 0, st>>>(x, M, K, x8, x8_pitch, dx);
+    if (operand_order) quantize_a8_kernel<true><<<(unsigned)M, (unsigned)threads, 0, st>>>(x, M, K, x8, x8_pitch, dx);
+    else quantize_a8_kernel<false><<<(unsigned)M, (unsigned)threads, 0, st>>>(x, M, K, x8, x8_pitch, dx);
     return cudaGetLastError();
 }
 
