@@ -22,8 +22,8 @@ Workspace plan_workspace(const Dims &d, int64_t M, int mode) {
     size_t off = 0;
     w.status_off = off; off += 256;  // first, so cq_gemm_status finds it without knowing the problem
     // arrival counters: one per 128-row block (small M) or per output tile (split-K GEMM)
-    const int64_t bnt = gemm_tc_token_tile(M);
-    const int sk = (M > 16 && mode == CQ_MODEL_DTYPE) ? gemm_tc_split_k(d, M) : 1;
+    const int64_t bnt = mode == CQ_MODEL_DTYPE ? gemm_tc_token_tile(M) : gemm_a8_token_tile(d, M);
+    const int sk = M <= 16 ? 1 : mode == CQ_MODEL_DTYPE ? gemm_tc_split_k(d, M) : gemm_a8_split_k(d, M);
     const size_t n_ctr = (size_t)d.NB * (M > 16 ? (size_t)((M + bnt - 1) / bnt) : 1);
     w.counters_off = off; w.counters_bytes = align_up(n_ctr * 4, 256); off += w.counters_bytes;
     size_t part = (size_t)gp.ctas * 2 * Mc * TILE * 4;   // two partial slots per CTA

@@ -20,6 +20,23 @@
 
 namespace cq {
 
+// Token tile of the Dynamic-A8 GEMM (two accumulator buffers of (128 / G) x tile columns fill at most
+// the 512 TMEM columns), and its split-K factor for grids that would leave most SMs idle.
+int gemm_a8_token_tile(const Dims &d, int64_t M) {
+    const int bmax = 256 / d.gpt;
+    const int bn = M <= 64 ? 64 : M <= 128 ? 128 : 256;
+    return bn < bmax ? bn : bmax;
+}
+int gemm_a8_split_k(const Dims &d, int64_t M) {
+    const int64_t bnt = gemm_a8_token_tile(d, M);
+    const int64_t ctas = (int64_t)d.NB * ((M + bnt - 1) / bnt);
+    if (ctas >= 100 || M > 256) return 1;
+    int64_t sk = 148 / ctas;
+    if (sk > 8) sk = 8;
+    if (sk > d.KT / 4) sk = d.KT / 4;   // at least four layout tiles per slice
+    return sk < 1 ? 1 : (int)sk;
+}
+
 namespace {
 
 using namespace tc;
@@ -39,6 +56,8 @@ struct A8Params {
     Dims d;
     int M;
     int raw_stage_bytes;
+    float *partial;       // split-K: fp32 partial sums [SK][M][Np] (before the d_x / 127 factor)
+    int *counters;        // split-K: arrival counters, one per (row block, token tile)
 };
 
 __device__ __forceinline__ void named_barrier_sync(int id, int threads) {
@@ -73,7 +92,9 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
     const Dims &d = prm.d;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nb = blockIdx.x, mt = blockIdx.y;
-    const int KT = d.KT;
+    // split-K: blockIdx.z takes the layout tiles [kt0, kt0 + KT) of the K range
+    const int kt0 = (int)(((int64_t)d.KT * blockIdx.z) / gridDim.z);
+    const int KT = (int)(((int64_t)d.KT * (blockIdx.z + 1)) / gridDim.z) - kt0;
 
     if ((smem_u32(smem) & 1023u) != 0) {
         if (threadIdx.x == 0) atomicCAS(prm.status, 0, 9);
@@ -98,7 +119,7 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
     if (warp == 0) {
         // ===== producer
         if (lane == 0) {
-            const uint8_t *tiles = prm.layout + (size_t)nb * KT * (size_t)d.tile_bytes;
+            const uint8_t *tiles = prm.layout + ((size_t)nb * d.KT + kt0) * (size_t)d.tile_bytes;
             bool ok = true;
             for (int t = 0; t < KT && ok; ++t) {
                 const int rs = t % A8_RAW_STAGES, s = t % A8_STAGES;
@@ -109,7 +130,7 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
                 if (t >= A8_STAGES) ok = mbar_wait(&st_empty[s], ((t / A8_STAGES) - 1) & 1, prm.status, 12);
                 if (!ok) break;
                 mbar_arrive_expect_tx(&b_full[s], B_STAGE_BYTES);
-                tma_load_2d(sB + s * B_STAGE_BYTES, &xmap, &b_full[s], t * 128, mt * BN);
+                tma_load_2d(sB + s * B_STAGE_BYTES, &xmap, &b_full[s], (kt0 + t) * 128, mt * BN);
             }
         }
     } else if (warp == 1) {
@@ -267,13 +288,17 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
         }
         if (ok) {
             const int64_t n = (int64_t)nb * TILE + drow;
-            if (n < d.N) {
+            if (n < d.N || gridDim.z > 1) {   // partial sums of padding channels are written too (zeros), never read back as y
 #pragma unroll
                 for (int i = 0; i < QCOLS; ++i) {
                     const int64_t m = (int64_t)mt * BN + cq4 * QCOLS + i;
                     if (m < prm.M) {
-                        const float v = acc[i] * (prm.dx[m] * (1.0f / 127.0f));
-                        prm.y[m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+                        if (gridDim.z == 1) {
+                            const float v = acc[i] * (prm.dx[m] * (1.0f / 127.0f));
+                            prm.y[m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+                        } else {
+                            prm.partial[((size_t)blockIdx.z * prm.M + m) * ((size_t)d.NB * TILE) + n] = acc[i];
+                        }
                     }
                 }
             }
@@ -286,13 +311,46 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+    if (gridDim.z > 1) {
+        // split-K combine: the last CTA of this output tile to arrive adds the slices in slice order and
+        // applies d_x / 127.  The barrier above ordered the CTA's partial stores before thread 0's release.
+        volatile int *s_last_p = reinterpret_cast<volatile int *>(tmem_slot + 1);   // scratch word after the TMEM slot
+        int *ctr = prm.counters + (nb * gridDim.y + mt);
+        if (threadIdx.x == 0) {
+            int old;
+            asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(ctr) : "memory");
+            *s_last_p = (old == (int)gridDim.z - 1);
+        }
+        __syncthreads();
+        if (*s_last_p) {
+            const size_t Np = (size_t)d.NB * TILE;
+            constexpr int QUADS = BN * TILE / 4;   // four consecutive channels of one token per 128-bit load
+            for (int qd = threadIdx.x; qd < QUADS; qd += A8_THREADS) {
+                const int64_t m = (int64_t)mt * BN + qd / (TILE / 4), n = (int64_t)nb * TILE + (qd % (TILE / 4)) * 4;
+                if (m >= prm.M) continue;
+                float4 v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    v[q] = q < (int)gridDim.z ? __ldcg(reinterpret_cast<const float4 *>(prm.partial + ((size_t)q * prm.M + m) * Np + n))
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+                float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) { sum.x += v[q].x; sum.y += v[q].y; sum.z += v[q].z; sum.w += v[q].w; }  // slice order
+                const float f = prm.dx[m] * (1.0f / 127.0f);
+                const float o[4] = {sum.x * f, sum.y * f, sum.z * f, sum.w * f};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (n + e < d.N) prm.y[m * d.N + n + e] = __bfloat16_as_ushort(__float2bfloat16_rn(o[e]));
+            }
+            if (threadIdx.x == 0) *ctr = 0;  // leave the workspace ready for the next call
+        }
+    }
 }
 
-template <int B, int G>
+template <int B, int G, int BN>
 cudaError_t launch_a8(const void *layout, const Dims &d, const int8_t *x8, int64_t pitch, const float *dx, uint16_t *y,
-                      int64_t M, int *status, cudaStream_t st) {
+                      int64_t M, int *status, float *partial, int *counters, cudaStream_t st) {
     constexpr int GPT = TILE / G;
-    constexpr int BN = 256 / GPT;   // two accumulator buffers of GPT x BN columns fill the 512 TMEM columns
     EncodeTiledFn enc = encode_tiled();
     if (!enc) return cudaErrorNotSupported;
     CUtensorMap xmap;
@@ -306,6 +364,7 @@ cudaError_t launch_a8(const void *layout, const Dims &d, const int8_t *x8, int64
         return cudaErrorInvalidValue;
     A8Params p;
     p.layout = (const uint8_t *)layout; p.dx = dx; p.y = y; p.status = status; p.d = d; p.M = (int)M;
+    p.partial = partial; p.counters = counters;
     p.raw_stage_bytes = (d.tile_bytes + 1023) / 1024 * 1024;
     const size_t smem = (size_t)A8_STAGES * (A8_A_STAGE_BYTES + BN * 128) + (size_t)A8_RAW_STAGES * p.raw_stage_bytes +
                         (size_t)8 * 2 * 16 * (1 << B) + (size_t)A8_SRING * 128 * GPT * 4 + 512 + 256;
@@ -316,18 +375,29 @@ cudaError_t launch_a8(const void *layout, const Dims &d, const int8_t *x8, int64
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    dim3 grid((unsigned)d.NB, (unsigned)((M + BN - 1) / BN));
+    dim3 grid((unsigned)d.NB, (unsigned)((M + BN - 1) / BN), (unsigned)gemm_a8_split_k(d, M));
     kern<<<grid, A8_THREADS, smem, st>>>(xmap, p);
     return cudaGetLastError();
 }
 
+// token tile: two accumulator buffers of GPT x BN columns must fit the 512 TMEM columns
+template <int B, int G>
+cudaError_t launch_a8_bn(const void *layout, const Dims &d, const int8_t *x8, int64_t pitch, const float *dx, uint16_t *y,
+                         int64_t M, int *status, float *partial, int *counters, cudaStream_t st) {
+    constexpr int BMAX = 256 / (TILE / G);
+    const int bn = gemm_a8_token_tile(d, M);
+    if constexpr (BMAX >= 256) if (bn == 256) return launch_a8<B, G, 256>(layout, d, x8, pitch, dx, y, M, status, partial, counters, st);
+    if constexpr (BMAX >= 128) if (bn == 128) return launch_a8<B, G, 128>(layout, d, x8, pitch, dx, y, M, status, partial, counters, st);
+    return launch_a8<B, G, 64>(layout, d, x8, pitch, dx, y, M, status, partial, counters, st);
+}
+
 template <int B>
 cudaError_t launch_a8_b(const void *layout, const Dims &d, const int8_t *x8, int64_t pitch, const float *dx, uint16_t *y,
-                        int64_t M, int *status, cudaStream_t st) {
+                        int64_t M, int *status, float *partial, int *counters, cudaStream_t st) {
     switch (d.G) {
-        case 32: return launch_a8<B, 32>(layout, d, x8, pitch, dx, y, M, status, st);
-        case 64: return launch_a8<B, 64>(layout, d, x8, pitch, dx, y, M, status, st);
-        default: return launch_a8<B, 128>(layout, d, x8, pitch, dx, y, M, status, st);
+        case 32: return launch_a8_bn<B, 32>(layout, d, x8, pitch, dx, y, M, status, partial, counters, st);
+        case 64: return launch_a8_bn<B, 64>(layout, d, x8, pitch, dx, y, M, status, partial, counters, st);
+        default: return launch_a8_bn<B, 128>(layout, d, x8, pitch, dx, y, M, status, partial, counters, st);
     }
 }
 
@@ -339,18 +409,20 @@ cudaError_t launch_gemm_a8_tc(const void *layout, const Dims &d, const uint16_t 
     int8_t *xq = reinterpret_cast<int8_t *>(ws + plan.x8_off);
     float *dxs = reinterpret_cast<float *>(ws + plan.dx_off);
     int *status = reinterpret_cast<int *>(ws + plan.status_off);
+    float *partial = reinterpret_cast<float *>(ws + plan.partial_off);
+    int *counters = reinterpret_cast<int *>(ws + plan.counters_off);
     const int64_t pitch = (int64_t)d.KT * TILE;
     cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, true, st);
     if (e != cudaSuccess) return e;
     switch (d.B) {
-        case 1: return launch_a8_b<1>(layout, d, xq, pitch, dxs, y, M, status, st);
-        case 2: return launch_a8_b<2>(layout, d, xq, pitch, dxs, y, M, status, st);
-        case 3: return launch_a8_b<3>(layout, d, xq, pitch, dxs, y, M, status, st);
-        case 4: return launch_a8_b<4>(layout, d, xq, pitch, dxs, y, M, status, st);
-        case 5: return launch_a8_b<5>(layout, d, xq, pitch, dxs, y, M, status, st);
-        case 6: return launch_a8_b<6>(layout, d, xq, pitch, dxs, y, M, status, st);
-        case 7: return launch_a8_b<7>(layout, d, xq, pitch, dxs, y, M, status, st);
-        default: return launch_a8_b<8>(layout, d, xq, pitch, dxs, y, M, status, st);
+        case 1: return launch_a8_b<1>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
+        case 2: return launch_a8_b<2>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
+        case 3: return launch_a8_b<3>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
+        case 4: return launch_a8_b<4>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
+        case 5: return launch_a8_b<5>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
+        case 6: return launch_a8_b<6>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
+        case 7: return launch_a8_b<7>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
+        default: return launch_a8_b<8>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
     }
 }
 

@@ -40,6 +40,8 @@ cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, ui
                         uint8_t *ws, const Workspace &plan, cudaStream_t st);
 int gemm_tc_token_tile(int64_t M);
 int gemm_tc_split_k(const Dims &d, int64_t M);
+int gemm_a8_token_tile(const Dims &d, int64_t M);
+int gemm_a8_split_k(const Dims &d, int64_t M);
 // Large-M tcgen05 / TMEM GEMM, both activation modes.
 cudaError_t launch_gemm_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
                            uint8_t *ws, const Workspace &plan, cudaStream_t st);
