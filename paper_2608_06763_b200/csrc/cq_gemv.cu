@@ -309,7 +309,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
             if constexpr (MODE == 0) {
                 __half *xs = reinterpret_cast<__half *>(smem);
                 // pass 1: row maxima of |x| (as bf16 bit patterns) from the chunks this thread copied
-                for (int m = 0; m < M; ++m) {
+                auto thread_max = [&](int m) -> unsigned {
                     unsigned mx = 0;
                     if (c < cpr) {
                         const uint4 v = *(const uint4 *)(xs + m * XS + c * 8);
@@ -317,13 +317,11 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
 #pragma unroll
                         for (int q = 0; q < 4; ++q) { mx = max(mx, ws[q] & 0x7FFFu); mx = max(mx, (ws[q] >> 16) & 0x7FFFu); }
                     }
-                    mx = __reduce_max_sync(0xffffffffu, mx);
-                    if (lane == 0 && mx) atomicMax(&s_max[m], mx);
-                }
-                __syncthreads();
+                    return mx;
+                };
                 // pass 2: every thread derives the power-of-two scale that puts the row maximum in
                 // [2^14, 2^15) and converts the chunks it owns
-                for (int m = 0; m < M; ++m) {
+                auto convert_row = [&](int m) {
                     const unsigned mb = s_max[m];
                     const int ef = (int)((mb >> 7) & 0xFF);          // biased exponent of the maximum
                     int sh = (mb == 0 || ef == 255) ? 0 : 14 - ef + 127;
@@ -340,6 +338,29 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                         }
                         *(uint4 *)(xs + m * XS + c * 8) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
                     }
+                };
+                if (M <= 2) {   // the common decode case: short plain loops
+                    for (int m = 0; m < M; ++m) {
+                        const unsigned mx = __reduce_max_sync(0xffffffffu, thread_max(m));
+                        if (lane == 0 && mx) atomicMax(&s_max[m], mx);
+                    }
+                    __syncthreads();
+                    for (int m = 0; m < M; ++m) convert_row(m);
+                } else {        // more rows: they are independent, so their loads, reductions and atomics overlap
+                    unsigned mxs[RT];
+#pragma unroll
+                    for (int m = 0; m < RT; ++m) mxs[m] = m < M ? thread_max(m) : 0u;
+#pragma unroll
+                    for (int m = 0; m < RT; ++m) {
+                        if (m < M) {
+                            const unsigned mx = __reduce_max_sync(0xffffffffu, mxs[m]);
+                            if (lane == 0 && mx) atomicMax(&s_max[m], mx);
+                        }
+                    }
+                    __syncthreads();
+#pragma unroll 4
+                    for (int m = 0; m < RT; ++m)
+                        if (m < M) convert_row(m);
                 }
             } else {
                 if (threadIdx.x < 16) s_inv[threadIdx.x] = threadIdx.x < M ? dxs[threadIdx.x] * (1.0f / 127.0f) : 0.0f;
@@ -411,21 +432,46 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                 const int c_first = owner_of(nb, 0, d.KT, E, V, P);   // its segment starts the row block: slot 0
                 const int n_contrib = owner_of(nb, d.KT - 1, d.KT, E, V, P) - c_first + 1;
                 const float *pb = partial + ((size_t)c_first * 2 + 1) * (size_t)(M * TILE);   // slot 1 of CTA c_first + q
-                for (int idx = threadIdx.x; idx < M * TILE; idx += GEMV_THREADS) {
-                    const int m = idx / TILE, r = idx % TILE;
-                    const int64_t n = (int64_t)nb * TILE + r;
-                    float sum = 0.0f;
-                    for (int q0 = 0; q0 < n_contrib; q0 += 8) {  // eight independent loads in flight, added in K order
-                        float v[8];
+                if (M <= 2) {
+                    for (int idx = threadIdx.x; idx < M * TILE; idx += GEMV_THREADS) {
+                        const int m = idx / TILE, r = idx % TILE;
+                        const int64_t n = (int64_t)nb * TILE + r;
+                        float sum = 0.0f;
+                        for (int q0 = 0; q0 < n_contrib; q0 += 8) {  // eight independent loads in flight, added in K order
+                            float v[8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const size_t off = (size_t)(q0 + i) * 2 * (M * TILE) - (q0 + i == 0 ? (size_t)(M * TILE) : 0);
-                            v[i] = (q0 + i < n_contrib) ? __ldcg(pb + off + idx) : 0.0f;
+                            for (int i = 0; i < 8; ++i) {
+                                const size_t off = (size_t)(q0 + i) * 2 * (M * TILE) - (q0 + i == 0 ? (size_t)(M * TILE) : 0);
+                                v[i] = (q0 + i < n_contrib) ? __ldcg(pb + off + idx) : 0.0f;
+                            }
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) sum += v[i];
                         }
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) sum += v[i];
+                        if (n < d.N) y[(int64_t)m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(sum));
                     }
-                    if (n < d.N) y[(int64_t)m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(sum));
+                } else {
+                    // four consecutive channels of one token per thread and step (128-bit loads), up to eight
+                    // slots in flight, added in K order
+                    for (int idx = threadIdx.x; idx < M * (TILE / 4); idx += GEMV_THREADS) {
+                        const int m = idx / (TILE / 4), r = (idx % (TILE / 4)) * 4;
+                        const int64_t n = (int64_t)nb * TILE + r;
+                        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int q0 = 0; q0 < n_contrib; q0 += 8) {
+                            float4 v[8];
+    #pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                const size_t off = (size_t)(q0 + i) * 2 * (M * TILE) - (q0 + i == 0 ? (size_t)(M * TILE) : 0);
+                                v[i] = (q0 + i < n_contrib) ? __ldcg(reinterpret_cast<const float4 *>(pb + off + m * TILE + r))
+                                                            : make_float4(0.f, 0.f, 0.f, 0.f);
+                            }
+    #pragma unroll
+                            for (int i = 0; i < 8; ++i) { sum.x += v[i].x; sum.y += v[i].y; sum.z += v[i].z; sum.w += v[i].w; }
+                        }
+                        const float o[4] = {sum.x, sum.y, sum.z, sum.w};
+    #pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if (n + e < d.N) y[(int64_t)m * d.N + n + e] = __bfloat16_as_ushort(__float2bfloat16_rn(o[e]));
+                    }
                 }
                 if (threadIdx.x == 0) counters[nb] = 0;  // leave the workspace ready for the next call
             }

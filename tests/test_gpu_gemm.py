@@ -149,3 +149,25 @@ def test_wide_groups_all_paths(B, G, M, mode):
     x = datagen.activations(M, 1024, seed=191, outlier_cols=0.01)
     y, ref = run_both(c, x, mode)
     check_y(y, ref, f"G={G} B={B} M={M} mode={mode}")
+
+
+@pytest.mark.parametrize("G", [64, 128])
+@pytest.mark.parametrize("M", [40, 100, 128, 200])
+def test_a8_gemm_token_tiles_and_split_k(M, G):
+    # few output tiles and a long K: the INT8 tcgen05 path picks its token tile from M (64 / 128 / 256,
+    # capped by the group count) and cuts K into slices combined in slice order; two calls on one
+    # workspace must agree bit for bit (arrival counters are left cleared)
+    N, K, B = 200, 2048, 4
+    c = logical_case(N, K, B, G, seed=190 + M)
+    c.k[7, 100:140] = -(1 << (B - 1))
+    c = Case(c.k, c.s, c.a, c.b, B, G)
+    x = datagen.activations(M, K, seed=191, outlier_cols=0.01)
+    y, ref = run_both(c, x, cq.CQ_DYN_A8)
+    check_y(y, ref, f"a8 split-K M={M} G={G}")
+    ws = torch.zeros(cq.cq_workspace_bytes(B, G, M, N, K, 1), dtype=torch.uint8, device="cuda")
+    xd = x_to_device(x)
+    y1 = cq.cq_gemm(c.pw, xd, 1, ws).clone()
+    y2 = cq.cq_gemm(c.pw, xd, 1, ws).clone()
+    assert cq.cq_gemm_status(ws) == 0
+    assert torch.equal(y1.view(torch.int16), y2.view(torch.int16))
+    assert np.array_equal(y_to_numpy(y1), y)
