@@ -47,6 +47,7 @@ def lib():
         L.cqo_double_to_half.restype = C.c_uint16
         L.cqo_double_to_half.argtypes = [C.c_double]
         L.cqo_group_sse.restype = C.c_double
+        L.cqo_joint_scale.restype = C.c_double
         L.cqo_gemm_a8.restype = C.c_int64
         L.cqo_num_threads.restype = C.c_int
         L.cqo_num_levels.restype = C.c_int
@@ -152,8 +153,9 @@ def unpack(codes: np.ndarray, K: int, B: int) -> np.ndarray:
 EFFORT = {"int_absmax": 0, "int_clipped": 1, "fast": 2, "reference": 3}
 
 
-def encode(W: np.ndarray, B: int, G: int, effort: str = "fast"):
-    """Groupwise encoder: returns (k int8 [N,K], s fp32 [N,K/G], a fp16, b fp16)."""
+def encode(W: np.ndarray, B: int, G: int, effort: str = "fast", objective: str = "continuous"):
+    """Groupwise encoder: returns (k int8 [N,K], s fp32 [N,K/G], a fp16, b fp16).
+    objective "continuous" minimises L_C (Section 4.1), "joint" L_C + L_A8 (Section 4.3)."""
     W = _c(W, np.float32)
     N, K = W.shape
     assert K % G == 0 and G <= 512
@@ -162,9 +164,51 @@ def encode(W: np.ndarray, B: int, G: int, effort: str = "fast"):
     s = np.zeros((N, ng), dtype=np.float32)
     a = np.zeros((N, ng), dtype=np.uint16)
     b = np.zeros((N, ng), dtype=np.uint16)
-    lib().cqo_encode(_p(W), C.c_int64(N), C.c_int64(K), C.c_int(B), C.c_int(G), C.c_int(EFFORT[effort]),
-                     _p(k), _p(s), _p(a), _p(b))
+    fn = {"continuous": lib().cqo_encode, "joint": lib().cqo_encode_joint}[objective]
+    fn(_p(W), C.c_int64(N), C.c_int64(K), C.c_int(B), C.c_int(G), C.c_int(EFFORT[effort]), _p(k), _p(s), _p(a), _p(b))
     return k, s, a.view(np.float16), b.view(np.float16)
+
+
+def joint_levels(B: int, a16, b16):
+    """(z, ztilde): continuous normalised levels q(i/M) and carrier-grid levels round(127 q)/127."""
+    n = num_levels(B)
+    z = np.zeros(n, dtype=np.float64)
+    zt = np.zeros(n, dtype=np.float64)
+    a16 = int(_h(np.array([a16]))[0])
+    b16 = int(_h(np.array([b16]))[0])
+    lib().cqo_joint_levels(C.c_int(B), C.c_uint16(a16), C.c_uint16(b16), _p(z), _p(zt))
+    return z, zt
+
+
+def assign_group_joint(w, B, s, a16, b16) -> np.ndarray:
+    w = _c(w, np.float32)
+    k = np.zeros(w.size, dtype=np.int8)
+    a16 = int(_h(np.array([a16]))[0])
+    b16 = int(_h(np.array([b16]))[0])
+    lib().cqo_assign_group_joint(_p(w), C.c_int(w.size), C.c_int(B), C.c_float(float(s)), C.c_uint16(a16),
+                                 C.c_uint16(b16), _p(k))
+    return k
+
+
+def group_losses(w, B, s, a16, b16, k):
+    """(L_C, L_A8) of one group for stored codes (Eq. continuous-and-carrier-loss)."""
+    w = _c(w, np.float32)
+    k = _c(k, np.int8)
+    a16 = int(_h(np.array([a16]))[0])
+    b16 = int(_h(np.array([b16]))[0])
+    lc, la = C.c_double(0.0), C.c_double(0.0)
+    lib().cqo_group_losses(_p(w), C.c_int(w.size), C.c_int(B), C.c_float(float(s)), C.c_uint16(a16), C.c_uint16(b16),
+                           _p(k), C.byref(lc), C.byref(la))
+    return lc.value, la.value
+
+
+def joint_scale(w, k, B, a16, b16) -> float:
+    """Scale minimising L_C + L_A8 for fixed codes and shape (Eq. carrier-aware-scale)."""
+    w = _c(w, np.float32)
+    k = _c(k, np.int8)
+    a16 = int(_h(np.array([a16]))[0])
+    b16 = int(_h(np.array([b16]))[0])
+    return lib().cqo_joint_scale(_p(w), _p(k), C.c_int(w.size), C.c_int(B), C.c_uint16(a16), C.c_uint16(b16))
 
 
 def assign_group(w, B, s, a16, b16) -> np.ndarray:

@@ -15,8 +15,11 @@
  * Pins (tests/test_oracle_*.py): uniform-INT special case, endpoint
  * identities, m(a,b) against a brute-force minimum, population distortion
  * tables and closed forms (python side), brute-force nearest level and
- * least-squares scale on tiny groups, storage size, A8 identities.
- * Parity unpinned: the *search* inside cqo_encode (candidate list, clip list,
+ * least-squares scale on tiny groups, storage size, A8 identities; for the
+ * carrier-aware objective of Section 4.3: enumeration of every code vector, the
+ * joint decision boundaries, stationarity of the joint loss in s, the W1 / W2 and
+ * integer-grid cases where the carrier projection is the identity.
+ * Parity unpinned: the *search* inside cqo_encode / cqo_encode_joint (candidate list, clip list,
  * iteration counts are this file's reading; several (codes, params) outputs are
  * valid for one input).  Its building blocks (assignment, scale) are pinned, and
  * its result is checked against invariants (never worse than clipped INT, never
@@ -257,6 +260,102 @@ CQO_API double cqo_group_sse(const float *w, int G, int B, float s, uint16_t a16
     return sse;
 }
 
+/* ------------------------------------------------------------------ carrier-aware fitting (Section 4.3) */
+
+/* Carrier-grid levels of a shape given in fp32: ztilde_i = r_i / 127 with r_i by the pinned
+ * sequence of cqo_carriers (Eq. carrier-grid).  W2: {0, 1}. */
+static void carrier_grid(int B, float a, float b, double *zt) {
+    int M = max_code(B);
+    if (B == 2) { zt[0] = 0.0; zt[1] = 1.0; return; }
+    float c = (1.0f - a) - b;
+    for (int i = 0; i <= M; ++i) {
+        float t = (float)i / (float)M;
+        float q = t * fmaf(t, fmaf(t, c, b), a);
+        int iv = (int)rintf(127.0f * q);
+        if (iv < 0) iv = 0;
+        if (iv > 127) iv = 127;
+        zt[i] = (double)iv / 127.0;
+    }
+}
+
+/* Normalised continuous levels z_i = q(i/M) and carrier-grid levels ztilde_i = round(127 z_i)/127
+ * of a serialised shape (Eq. carrier-grid; z in fp64, the rounding by the pinned carrier sequence). */
+CQO_API void cqo_joint_levels(int B, uint16_t a16, uint16_t b16, double *z, double *zt) {
+    int M = max_code(B);
+    double a = half_to_double(a16), b = half_to_double(b16);
+    for (int i = 0; i <= M; ++i) z[i] = curve((double)i / (double)M, a, b);
+    carrier_grid(B, (float)a, (float)b, zt);
+}
+
+/* Magnitude index minimising (u - s z_i)^2 + (u - s ztilde_i)^2 over i = 0..M
+ * (Eq. carrier-aware-assignment), by plain scan; ties go to the lower index. */
+static int joint_index(double u, double s, const double *z, const double *zt, int M) {
+    int best = 0;
+    double bc = INFINITY;
+    for (int i = 0; i <= M; ++i) {
+        double d1 = u - s * z[i], d2 = u - s * zt[i];
+        double cst = d1 * d1 + d2 * d2;
+        if (cst < bc) { bc = cst; best = i; }
+    }
+    return best;
+}
+
+/* Codes of one group for fixed serialised parameters under the joint objective
+ * (Eq. carrier-aware-assignment).  W1: sign only. */
+CQO_API void cqo_assign_group_joint(const float *w, int G, int B, float s, uint16_t a16, uint16_t b16, int8_t *k) {
+    if (B == 1) { for (int j = 0; j < G; ++j) k[j] = (int8_t)(w[j] >= 0.0f ? 1 : -1); return; }
+    int M = max_code(B);
+    double z[128], zt[128];
+    cqo_joint_levels(B, a16, b16, z, zt);
+    for (int j = 0; j < G; ++j) {
+        int i = joint_index(fabs((double)w[j]), (double)s, z, zt, M);
+        k[j] = (int8_t)(w[j] < 0.0f ? -i : i);
+    }
+}
+
+/* The two groupwise squared errors of Eq. continuous-and-carrier-loss for stored codes:
+ * L_C against s q(t_k) and L_A8 against (s / 127) r(k). */
+CQO_API void cqo_group_losses(const float *w, int G, int B, float s, uint16_t a16, uint16_t b16, const int8_t *k,
+                              double *LC, double *LA8) {
+    double lc = 0.0, la = 0.0;
+    if (B == 1) {
+        for (int j = 0; j < G; ++j) { double d = (double)w[j] - (k[j] > 0 ? 1.0 : -1.0) * (double)s; lc += d * d; }
+        *LC = lc; *LA8 = lc; return;
+    }
+    double z[128], zt[128];
+    cqo_joint_levels(B, a16, b16, z, zt);
+    for (int j = 0; j < G; ++j) {
+        int kk = k[j], i = kk < 0 ? -kk : kk;
+        double sg = kk < 0 ? -1.0 : 1.0;
+        if (kk == -(1 << (B - 1))) { i = 0; } /* reserved pattern decodes to zero */
+        double d1 = (double)w[j] - sg * (double)s * z[i], d2 = (double)w[j] - sg * (double)s * zt[i];
+        lc += d1 * d1; la += d2 * d2;
+    }
+    *LC = lc; *LA8 = la;
+}
+
+/* Shared scale minimising L_C + L_A8 for fixed codes and shape (Eq. carrier-aware-scale):
+ * s* = sum u_j (z_j + ztilde_j) / sum (z_j^2 + ztilde_j^2); 0 when the denominator vanishes. */
+CQO_API double cqo_joint_scale(const float *w, const int8_t *k, int G, int B, uint16_t a16, uint16_t b16) {
+    if (B == 1) { double su = 0.0; for (int j = 0; j < G; ++j) su += fabs((double)w[j]); return su / G; }
+    double z[128], zt[128], num = 0.0, den = 0.0;
+    cqo_joint_levels(B, a16, b16, z, zt);
+    for (int j = 0; j < G; ++j) {
+        int kk = k[j], i = kk < 0 ? -kk : kk;
+        if (kk == -(1 << (B - 1))) i = 0;
+        double u = fabs((double)w[j]);
+        num += u * (z[i] + zt[i]);
+        den += z[i] * z[i] + zt[i] * zt[i];
+    }
+    return den > 0.0 ? num / den : 0.0;
+}
+
+static double joint_ls_scale(const double *u, const int *idx, int G, const double *z, const double *zt, double fallback) {
+    double num = 0.0, den = 0.0;
+    for (int j = 0; j < G; ++j) { int i = idx[j]; num += u[j] * (z[i] + zt[i]); den += z[i] * z[i] + zt[i] * zt[i]; }
+    return den > 0.0 ? num / den : fallback;
+}
+
 /* Least-squares scale for fixed magnitude indices and shape:  s = sum u_j z_j / sum z_j^2
  * with z_j = q(t_{i_j})  (the continuous-only analogue of Eq. carrier-aware-scale). */
 static double ls_scale(const double *u, const int *idx, int G, const double *z, double fallback) {
@@ -300,24 +399,26 @@ typedef struct {
  * increasing discrete levels), repeat the assignment under the rounded parameters,
  * re-fit and re-round the scale once, and return the squared error of what is stored. */
 static fit_t serialise_and_score(const float *w, const double *u, int G, int B, double s, double a, double b,
-                                 int8_t *kbuf) {
+                                 int8_t *kbuf, int joint) {
     fit_t f; f.valid = 0; f.sse = INFINITY; f.s = 0; f.a16 = 0; f.b16 = 0;
     int M = max_code(B);
     uint16_t a16 = double_to_half(a), b16 = double_to_half(b);
     double ar = half_to_double(a16), br = half_to_double(b16);
     if (!(s > 0.0) || !isfinite(s)) return f;
     if (!(cqo_shape_margin(ar, br) > 0.0)) return f;
-    double z[128];
+    double z[128], zt[128];
     for (int i = 0; i <= M; ++i) z[i] = curve((double)i / (double)M, ar, br);
     for (int i = 0; i < M; ++i) if (!(z[i + 1] > z[i])) return f;
+    if (joint) carrier_grid(B, (float)ar, (float)br, zt);
     int idx[512];
     double y[128];
     float s32 = (float)s;
     for (int pass = 0; pass < 2; ++pass) {
         for (int i = 0; i <= M; ++i) y[i] = (double)s32 * z[i];
-        for (int j = 0; j < G; ++j) idx[j] = nearest_index(u[j], y, M);
+        if (joint) for (int j = 0; j < G; ++j) idx[j] = joint_index(u[j], (double)s32, z, zt, M);
+        else for (int j = 0; j < G; ++j) idx[j] = nearest_index(u[j], y, M);
         if (pass == 0) {
-            double s2 = ls_scale(u, idx, G, z, (double)s32);
+            double s2 = joint ? joint_ls_scale(u, idx, G, z, zt, (double)s32) : ls_scale(u, idx, G, z, (double)s32);
             if (s2 > 0.0 && isfinite(s2)) s32 = (float)s2;
         }
     }
@@ -326,6 +427,7 @@ static fit_t serialise_and_score(const float *w, const double *u, int G, int B, 
     for (int j = 0; j < G; ++j) {
         double d = u[j] - y[idx[j]];
         sse += d * d;
+        if (joint) { double d2 = u[j] - (double)s32 * zt[idx[j]]; sse += d2 * d2; }  /* L_C + L_A8 */
         kbuf[j] = (int8_t)(w[j] < 0.0f ? -idx[j] : idx[j]);
     }
     f.valid = 1; f.sse = sse; f.s = s32; f.a16 = a16; f.b16 = b16;
@@ -339,19 +441,33 @@ static fit_t serialise_and_score(const float *w, const double *u, int G, int B, 
  * (s, s a, s b), so the squared error is minimised by 3x3 normal equations; a step is kept
  * only while the curve stays strictly monotone (m(a, b) > margin). */
 static void run_candidate(const float *w, const double *u, int G, int B, double a, double b, double s0,
-                          int iters, int refine, fit_t *best, int8_t *kbest, int8_t *kbuf) {
+                          int iters, int refine, fit_t *best, int8_t *kbest, int8_t *kbuf, int joint) {
     int M = max_code(B);
-    double z[128], y[128];
+    double z[128], y[128], zt[128];
     int idx[512];
     double s = s0;
+    /* joint objective (Section 4.3): the same candidates and the same refinement proposals, but the
+     * assignment is Eq. carrier-aware-assignment, the scale Eq. carrier-aware-scale, and the score
+     * L_C + L_A8; the carrier grid of an unserialised shape is taken from its fp32 value */
     for (int it = 0; it < iters; ++it) {
         for (int i = 0; i <= M; ++i) { z[i] = curve((double)i / (double)M, a, b); y[i] = s * z[i]; }
-        for (int j = 0; j < G; ++j) idx[j] = nearest_index(u[j], y, M);
-        s = ls_scale(u, idx, G, z, s);
+        if (joint) {
+            carrier_grid(B, (float)a, (float)b, zt);
+            for (int j = 0; j < G; ++j) idx[j] = joint_index(u[j], s, z, zt, M);
+            s = joint_ls_scale(u, idx, G, z, zt, s);
+        } else {
+            for (int j = 0; j < G; ++j) idx[j] = nearest_index(u[j], y, M);
+            s = ls_scale(u, idx, G, z, s);
+        }
     }
     for (int rf = 0; rf < refine; ++rf) {
         for (int i = 0; i <= M; ++i) { z[i] = curve((double)i / (double)M, a, b); y[i] = s * z[i]; }
-        for (int j = 0; j < G; ++j) idx[j] = nearest_index(u[j], y, M);
+        if (joint) {
+            carrier_grid(B, (float)a, (float)b, zt);
+            for (int j = 0; j < G; ++j) idx[j] = joint_index(u[j], s, z, zt, M);
+        } else {
+            for (int j = 0; j < G; ++j) idx[j] = nearest_index(u[j], y, M);
+        }
         double A[3][3] = {{0}}, r[3] = {0}, p[3];
         for (int j = 0; j < G; ++j) {
             double t = (double)idx[j] / (double)M, t2 = t * t, t3 = t2 * t;
@@ -368,7 +484,7 @@ static void run_candidate(const float *w, const double *u, int G, int B, double 
         if (fabs(an) > 8.0 || fabs(bn) > 8.0) break;
         s = p[0]; a = an; b = bn;
     }
-    fit_t f = serialise_and_score(w, u, G, B, s, a, b, kbuf);
+    fit_t f = serialise_and_score(w, u, G, B, s, a, b, kbuf, joint);
     if (f.valid && f.sse < best->sse) { /* strict: ties keep the earlier candidate */
         *best = f;
         memcpy(kbest, kbuf, (size_t)G);
@@ -403,7 +519,7 @@ static int build_shapes(int effort, double (*out)[2]) {
  *   2  fast: the candidates of 1, then 12 shapes x 3 clips, 3 assignment/scale rounds, 8 refinement rounds
  *   3  reference: the candidates of 1, then a dense shape grid x 6 clips, 4 assignment/scale rounds,
  *      12 refinement rounds */
-static void encode_group(const float *w, int G, int B, int effort, int8_t *k, float *s_out, uint16_t *a_out,
+static void encode_group(const float *w, int G, int B, int effort, int joint, int8_t *k, float *s_out, uint16_t *a_out,
                          uint16_t *b_out) {
     const uint16_t ONE16 = 0x3C00;
     double u[512], umax = 0.0, usum = 0.0;
@@ -442,10 +558,18 @@ static void encode_group(const float *w, int G, int B, int effort, int8_t *k, fl
      * worse than clipped INT under the same objective (Section 2.2, after Eq. int-special-case) */
     if (effort >= 2)
         for (int ci = 0; ci < 15; ++ci)
-            run_candidate(w, u, G, B, 1.0, 0.0, clips_int[ci] * umax, 6, 0, &best, k, kbuf);
+            run_candidate(w, u, G, B, 1.0, 0.0, clips_int[ci] * umax, 6, 0, &best, k, kbuf, joint);
     for (int si = 0; si < ns; ++si)
         for (int ci = 0; ci < nc; ++ci)
-            run_candidate(w, u, G, B, shapes[si][0], shapes[si][1], clips[ci] * umax, iters, refine, &best, k, kbuf);
+            run_candidate(w, u, G, B, shapes[si][0], shapes[si][1], clips[ci] * umax, iters, refine, &best, k, kbuf, joint);
+    if (joint && effort >= 1 && B > 2) {
+        /* the continuous fitter's own answer also competes, re-scored under the joint objective, so the
+         * carrier-aware result is never worse (jointly) than the continuous-only one */
+        int8_t kc[512]; float sc; uint16_t ac, bc;
+        encode_group(w, G, B, effort, 0, kc, &sc, &ac, &bc);
+        fit_t f = serialise_and_score(w, u, G, B, (double)sc, half_to_double(ac), half_to_double(bc), kbuf, 1);
+        if (f.valid && f.sse < best.sse) { best = f; memcpy(k, kbuf, (size_t)G); }
+    }
     if (!best.valid) { /* cannot happen for finite input; keep absmax INT */
         float s32 = (float)umax;
         cqo_assign_group(w, G, B, s32, ONE16, 0, k);
@@ -463,7 +587,19 @@ CQO_API void cqo_encode(const float *W, int64_t N, int64_t K, int B, int G, int 
 #pragma omp parallel for schedule(dynamic, 64)
     for (int64_t gi = 0; gi < N * ng; ++gi) {
         int64_t n = gi / ng, g = gi % ng;
-        encode_group(W + n * K + g * G, G, B, effort, k + n * K + g * G, &s[gi], &a[gi], &b[gi]);
+        encode_group(W + n * K + g * G, G, B, effort, 0, k + n * K + g * G, &s[gi], &a[gi], &b[gi]);
+    }
+}
+
+/* The same search under the dual-path objective L_C + L_A8 of Section 4.3 (effort 0, the absmax INT
+ * pin, is objective-free).  For W1 / W2 the levels lie on the carrier grid, so the result equals cqo_encode's. */
+CQO_API void cqo_encode_joint(const float *W, int64_t N, int64_t K, int B, int G, int effort, int8_t *k, float *s,
+                              uint16_t *a, uint16_t *b) {
+    int64_t ng = K / G;
+#pragma omp parallel for schedule(dynamic, 64)
+    for (int64_t gi = 0; gi < N * ng; ++gi) {
+        int64_t n = gi / ng, g = gi % ng;
+        encode_group(W + n * K + g * G, G, B, effort, B > 2 ? 1 : 0, k + n * K + g * G, &s[gi], &a[gi], &b[gi]);
     }
 }
 
