@@ -149,6 +149,34 @@ int cq_decode_weights(const void *layout, int B, int G, int64_t N, int64_t K, fl
 int cq_debug_a8_partials(const void *layout, int B, int G, const int8_t *x8, int64_t M, int64_t N, int64_t K,
                          int32_t *P, void *stream);
 
+/* ---- Offline encoder (the step before the hot path; Sections 4.1 and 4.3) --------------------------
+ * W[N][K] float, logical signed codes k[N][K] int8 (what cq_pack_codes takes), scale[N][K/G] float,
+ * a / b [N][K/G] binary16 bit patterns; all device pointers owned by the caller; nothing is allocated
+ * and nothing synchronises.  objective: CQ_FIT_CONTINUOUS minimises L_C = sum (w - s q)^2
+ * (Eq. offline-objective), CQ_FIT_JOINT minimises L_C + L_A8 with L_A8 taken against the INT8 carrier
+ * (s / 127) r(k) (Eq. carrier-aware-objective); for B <= 2 the two coincide.  Decisions are taken in
+ * fp64.  Errors: CQ_ERR_INVALID_ARG (null pointer, sizes <= 0, B outside 1..8, unknown objective or
+ * effort), CQ_ERR_UNSUPPORTED (K % G != 0 or G > 512), CQ_ERR_CUDA. */
+#define CQ_FIT_CONTINUOUS 0
+#define CQ_FIT_JOINT 1
+/* Codes for fixed stored parameters: nearest reconstruction level (Section 4.1), or the minimiser of
+ * (u - s q)^2 + (u - s qtilde)^2 (Eq. carrier-aware-assignment); ties go to the smaller magnitude; the
+ * reserved pattern is never produced; W1: the sign of w (w >= 0 -> +1). */
+int cq_encode_assign(const float *W, int B, int G, int64_t N, int64_t K, const float *scale, const uint16_t *a,
+                     const uint16_t *b, int objective, int8_t *k, void *stream);
+/* Scale for fixed codes and shape: sum u z / sum z^2, or Eq. carrier-aware-scale; 0 for an all-zero group. */
+int cq_encode_scale(const float *W, const int8_t *k, int B, int G, int64_t N, int64_t K, const uint16_t *a,
+                    const uint16_t *b, int objective, float *scale, void *stream);
+/* The two groupwise squared errors of Eq. continuous-and-carrier-loss: LC[N][K/G], LA8[N][K/G] double. */
+int cq_encode_losses(const float *W, const int8_t *k, int B, int G, int64_t N, int64_t K, const float *scale,
+                     const uint16_t *a, const uint16_t *b, double *LC, double *LA8, void *stream);
+/* The whole groupwise encoder: a deterministic search over monotone shape candidates and soft clips
+ * with alternating assignment / scale updates and a refinement of (s, a, b) by normal equations
+ * (Eq. affine-cubic-level), scored on what is stored (a, b in binary16, s in binary32, assignment
+ * repeated).  effort: 0 symmetric absmax integer grid, 1 clipped integer grid, 2 fast, 3 reference. */
+int cq_encode(const float *W, int B, int G, int64_t N, int64_t K, int objective, int effort, int8_t *k, float *scale,
+              uint16_t *a, uint16_t *b, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -59,9 +59,13 @@ def lib():
         L.cq_decode_carriers.argtypes = [vp, i, i, i64, i64, vp, vp]
         L.cq_decode_weights.argtypes = [vp, i, i, i64, i64, vp, vp]
         L.cq_debug_a8_partials.argtypes = [vp, i, i, vp, i64, i64, i64, vp, vp]
+        L.cq_encode_assign.argtypes = [vp, i, i, i64, i64, vp, vp, vp, i, vp, vp]
+        L.cq_encode_scale.argtypes = [vp, vp, i, i, i64, i64, vp, vp, i, vp, vp]
+        L.cq_encode_losses.argtypes = [vp, vp, i, i, i64, i64, vp, vp, vp, vp, vp, vp]
+        L.cq_encode.argtypes = [vp, i, i, i64, i64, i, i, vp, vp, vp, vp, vp]
         for name in ("cq_workspace_init", "cq_pack_codes", "cq_repack", "cq_unpack", "cq_gemm", "cq_gemm_host",
                      "cq_quantize_a8", "cq_decode_levels", "cq_decode_carriers", "cq_decode_weights",
-                     "cq_debug_a8_partials"):
+                     "cq_debug_a8_partials", "cq_encode_assign", "cq_encode_scale", "cq_encode_losses", "cq_encode"):
             getattr(L, name).restype = i
         _lib = L
     return _lib
@@ -226,3 +230,46 @@ def cq_debug_a8_partials(pw: PackedWeights, x8: torch.Tensor) -> torch.Tensor:
     _check(lib().cq_debug_a8_partials(_ptr(pw.layout), pw.B, pw.G, _ptr(x8), M, pw.N, pw.K, _ptr(out), _stream()),
            "cq_debug_a8_partials")
     return out
+
+
+CQ_FIT_CONTINUOUS, CQ_FIT_JOINT = 0, 1
+CQ_EFFORT = {"int_absmax": 0, "int_clipped": 1, "fast": 2, "reference": 3}
+
+
+def cq_encode_assign(W: torch.Tensor, B: int, G: int, scale, a, b, objective: int = CQ_FIT_CONTINUOUS) -> torch.Tensor:
+    """W float32 [N, K]; scale float32, a / b float16 [N, K/G] -> signed codes int8 [N, K]."""
+    N, K = W.shape
+    k = torch.empty((N, K), dtype=torch.int8, device=W.device)
+    _check(lib().cq_encode_assign(_ptr(W), B, G, N, K, _ptr(scale), _ptr(a), _ptr(b), objective, _ptr(k), _stream()),
+           "cq_encode_assign")
+    return k
+
+
+def cq_encode_scale(W: torch.Tensor, k: torch.Tensor, B: int, G: int, a, b, objective: int = CQ_FIT_CONTINUOUS) -> torch.Tensor:
+    N, K = W.shape
+    scale = torch.empty((N, K // G), dtype=torch.float32, device=W.device)
+    _check(lib().cq_encode_scale(_ptr(W), _ptr(k), B, G, N, K, _ptr(a), _ptr(b), objective, _ptr(scale), _stream()),
+           "cq_encode_scale")
+    return scale
+
+
+def cq_encode_losses(W: torch.Tensor, k: torch.Tensor, B: int, G: int, scale, a, b):
+    """(L_C, L_A8) float64 [N, K/G] of stored codes and parameters."""
+    N, K = W.shape
+    lc = torch.empty((N, K // G), dtype=torch.float64, device=W.device)
+    la = torch.empty_like(lc)
+    _check(lib().cq_encode_losses(_ptr(W), _ptr(k), B, G, N, K, _ptr(scale), _ptr(a), _ptr(b), _ptr(lc), _ptr(la),
+                                  _stream()), "cq_encode_losses")
+    return lc, la
+
+
+def cq_encode(W: torch.Tensor, B: int, G: int, objective: int = CQ_FIT_CONTINUOUS, effort: str = "fast"):
+    """The groupwise encoder: (k int8 [N, K], scale float32, a float16, b float16 [N, K/G])."""
+    N, K = W.shape
+    k = torch.empty((N, K), dtype=torch.int8, device=W.device)
+    scale = torch.empty((N, K // G), dtype=torch.float32, device=W.device)
+    a = torch.empty((N, K // G), dtype=torch.float16, device=W.device)
+    b = torch.empty_like(a)
+    _check(lib().cq_encode(_ptr(W), B, G, N, K, objective, CQ_EFFORT[effort], _ptr(k), _ptr(scale), _ptr(a), _ptr(b),
+                           _stream()), "cq_encode")
+    return k, scale, a, b

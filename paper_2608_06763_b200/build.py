@@ -17,10 +17,14 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libcubicquant.so")
-SOURCES = ["cq_api.cu", "cq_layout.cu", "cq_gemv.cu", "cq_gemm_tc.cu", "cq_gemm_a8_tc.cu", "cq_static.cu"]
+SOURCES = ["cq_api.cu", "cq_layout.cu", "cq_gemv.cu", "cq_gemm_tc.cu", "cq_gemm_a8_tc.cu", "cq_static.cu", "cq_encode.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr",
               "-I", INCLUDE, "-I", CSRC]
+
+
+# the encoder takes its decisions in fp64 as written: no contraction of a product and a sum into an FMA
+EXTRA_FLAGS = {"cq_encode.cu": ["-fmad=false"]}
 
 
 def _nvcc() -> str:
@@ -37,7 +41,7 @@ def _deps_mtime() -> float:
 
 def _compile(src: str, verbose: bool) -> str:
     obj = os.path.join(OBJ, src.replace(".cu", ".o"))
-    cmd = [_nvcc(), *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
+    cmd = [_nvcc(), *NVCC_FLAGS, *EXTRA_FLAGS.get(src, []), "-c", os.path.join(CSRC, src), "-o", obj]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     res = subprocess.run(cmd, capture_output=True, text=True)

@@ -180,6 +180,45 @@ int cq_gemm_host(const void *layout, int B, int G, const uint16_t *x_host, uint1
     return wrap(cudaStreamSynchronize(s));
 }
 
+static int check_encode(int B, int G, int64_t N, int64_t K, int objective) {
+    if (B < 1 || B > 8 || N <= 0 || K <= 0 || G <= 0) return CQ_ERR_INVALID_ARG;
+    if (objective != CQ_FIT_CONTINUOUS && objective != CQ_FIT_JOINT) return CQ_ERR_INVALID_ARG;
+    if (K % G != 0 || G > 512) return CQ_ERR_UNSUPPORTED;
+    return CQ_OK;
+}
+
+int cq_encode_assign(const float *W, int B, int G, int64_t N, int64_t K, const float *scale, const uint16_t *a,
+                     const uint16_t *b, int objective, int8_t *k, void *stream) {
+    if (!W || !scale || !a || !b || !k) return CQ_ERR_INVALID_ARG;
+    const int st = check_encode(B, G, N, K, objective);
+    if (st != CQ_OK) return st;
+    return wrap(launch_encode_assign(W, B, G, N, K, scale, a, b, objective, k, (cudaStream_t)stream));
+}
+
+int cq_encode_scale(const float *W, const int8_t *k, int B, int G, int64_t N, int64_t K, const uint16_t *a,
+                    const uint16_t *b, int objective, float *scale, void *stream) {
+    if (!W || !scale || !a || !b || !k) return CQ_ERR_INVALID_ARG;
+    const int st = check_encode(B, G, N, K, objective);
+    if (st != CQ_OK) return st;
+    return wrap(launch_encode_scale(W, k, B, G, N, K, a, b, objective, scale, (cudaStream_t)stream));
+}
+
+int cq_encode_losses(const float *W, const int8_t *k, int B, int G, int64_t N, int64_t K, const float *scale,
+                     const uint16_t *a, const uint16_t *b, double *LC, double *LA8, void *stream) {
+    if (!W || !scale || !a || !b || !k || !LC || !LA8) return CQ_ERR_INVALID_ARG;
+    const int st = check_encode(B, G, N, K, CQ_FIT_JOINT);
+    if (st != CQ_OK) return st;
+    return wrap(launch_encode_losses(W, k, B, G, N, K, scale, a, b, LC, LA8, (cudaStream_t)stream));
+}
+
+int cq_encode(const float *W, int B, int G, int64_t N, int64_t K, int objective, int effort, int8_t *k, float *scale,
+              uint16_t *a, uint16_t *b, void *stream) {
+    if (!W || !scale || !a || !b || !k || effort < 0 || effort > 3) return CQ_ERR_INVALID_ARG;
+    const int st = check_encode(B, G, N, K, objective);
+    if (st != CQ_OK) return st;
+    return wrap(launch_encode_search(W, B, G, N, K, objective, effort, k, scale, a, b, (cudaStream_t)stream));
+}
+
 int cq_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, float *dx, void *stream) {
     if (!x || !x8 || !dx || M <= 0 || K <= 0) return CQ_ERR_INVALID_ARG;
     return wrap(launch_quantize_a8(x, M, K, x8, K, dx, false, (cudaStream_t)stream));

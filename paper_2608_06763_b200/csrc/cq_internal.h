@@ -42,6 +42,16 @@ int gemm_tc_token_tile(int64_t M);
 int gemm_tc_split_k(const Dims &d, int64_t M);
 int gemm_a8_token_tile(const Dims &d, int64_t M);
 int gemm_a8_split_k(const Dims &d, int64_t M);
+
+// offline encoder steps (cq_encode.cu)
+cudaError_t launch_encode_assign(const float *W, int B, int G, int64_t N, int64_t K, const float *scale, const uint16_t *a,
+                                 const uint16_t *b, int joint, int8_t *k, cudaStream_t st);
+cudaError_t launch_encode_scale(const float *W, const int8_t *k, int B, int G, int64_t N, int64_t K, const uint16_t *a,
+                                const uint16_t *b, int joint, float *scale, cudaStream_t st);
+cudaError_t launch_encode_losses(const float *W, const int8_t *k, int B, int G, int64_t N, int64_t K, const float *scale,
+                                 const uint16_t *a, const uint16_t *b, double *LC, double *LA8, cudaStream_t st);
+cudaError_t launch_encode_search(const float *W, int B, int G, int64_t N, int64_t K, int joint, int effort, int8_t *k,
+                                 float *scale, uint16_t *a, uint16_t *b, cudaStream_t st);
 // Large-M tcgen05 / TMEM GEMM, both activation modes.
 cudaError_t launch_gemm_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
                            uint8_t *ws, const Workspace &plan, cudaStream_t st);

@@ -84,7 +84,7 @@ def test_joint_assignment_follows_the_joint_boundaries(B):
 def test_joint_scale_is_the_stationary_point_of_the_joint_loss(B):
     # Eq. carrier-aware-scale against the loss itself: L(s*) <= L(s* (1 +- eps)) and the central
     # difference of L at s* vanishes
-    W = datagen.weights("laplace", 4, 128, seed=21, scale=0.015)
+    W = datagen.weights("laplace", 4, 128, seed=21, b=0.015)
     a16, b16 = np.float16(0.6), np.float16(-0.25)
     for row in W:
         w = row.astype(np.float32)
@@ -138,7 +138,7 @@ def test_joint_encoder_invariants(B):
     # curves strictly monotone; (4) its A8 error is not larger than the continuous answer's by more than
     # the continuous error it gives up: L_joint(joint) <= L_joint(cont)
     G = 64
-    W = datagen.weights("laplace", 12, 256, seed=51, scale=0.015)
+    W = datagen.weights("laplace", 12, 256, seed=51, b=0.015)
     kc, sc, ac, bc = oracle.encode(W, B, G, "fast")
     kj, sj, aj, bj = oracle.encode(W, B, G, "fast", objective="joint")
     M = (1 << (B - 1)) - 1
