@@ -232,6 +232,22 @@ def extra_suites(torch, cq, datagen, stream, peaks):
                               "a16_over_a8": round(t[0] / t[1], 3)})
             del pw, cp
             torch.cuda.empty_cache()
+    # ---- offline encoder (the step before the hot path): 4096 x 4096, W4 G128, fast effort, both objectives
+    enc = []
+    Wd = torch.from_numpy(datagen.weights("normal", 4096, 4096, seed=0, sigma=0.02)).cuda()
+    for oname, obj in (("continuous", cq.CQ_FIT_CONTINUOUS), ("joint", cq.CQ_FIT_JOINT)):
+        cq.cq_encode(Wd[:256], 4, 128, obj, "fast")
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        cq.cq_encode(Wd, 4, 128, obj, "fast")
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        enc.append({"N": 4096, "K": 4096, "B": 4, "G": 128, "objective": oname, "effort": "fast", "ms": round(ms, 2),
+                    "mweights_per_s": round(4096 * 4096 / ms / 1e3, 1)})
+    del Wd
+    out["encoder_gpu"] = enc
     out["paper_h200_shapes_on_b200"] = paper
     out["decode_linears_w4g128"] = dec
     out["crossover"] = cross
