@@ -226,6 +226,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
     constexpr int RT = 8 * NT;       // staged token rows (rows >= M are zero)
     constexpr int NBUF = (B <= 4) ? 3 : 2;
     constexpr int ES = MODE == 0 ? 2 : 1;  // bytes per staged activation element
+    constexpr int CB = 2048 * B, TB = CB + 1024 * GPT;   // bytes of a tile's code part and of a whole tile
     constexpr int XPAD = MODE == 0 ? XS_PAD : XS_PAD8;
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ float s_inv[16];
@@ -258,9 +259,9 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
             const int ke = min(kb_end, ks + MAX_SUB);
             const int slice_k = (ke - ks) * TILE, XS = slice_k + XPAD;
             const int64_t k_base = (int64_t)ks * TILE;
-            const uint8_t *tile0 = layout + ((size_t)nb * d.KT + ks) * (size_t)d.tile_bytes;
+            const uint8_t *tile0 = layout + ((size_t)nb * d.KT + ks) * (size_t)TB;
             const uint8_t *wl = tile0 + warp * 256 * B + lane * 16;                     // next tile to load (codes)
-            const uint8_t *pl = tile0 + d.code_bytes + ((warp * 16 + g) * GPT) * 8;      // next tile to load (params)
+            const uint8_t *pl = tile0 + CB + ((warp * 16 + g) * GPT) * 8;      // next tile to load (params)
 
             // The activations, the workspace and y may be produced or still used by the kernel launched
             // before this one: wait for it (a no-op unless the launch allowed programmatic overlap), then
@@ -299,11 +300,9 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
             TileRegs<B, GPT> buf[NBUF];
             static_for<NBUF>([&](auto ic) {
                 constexpr int i = decltype(ic)::value;
-                if (ks + i < ke) {
-                    load_tile<B, GPT>(buf[i], wl, pl, lane);
-                    wl += d.tile_bytes; pl += d.tile_bytes;
-                }
+                if (ks + i < ke) load_tile<B, GPT>(buf[i], wl + i * TB, pl + i * TB, lane);
             });
+            wl += NBUF * TB; pl += NBUF * TB;   // tile offsets inside a round of NBUF loads are immediates
 
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             if constexpr (MODE == 0) {
@@ -383,12 +382,12 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                         compute_tile<B, G, NT, MODE>(buf[i], xcur, XS, ctab, g, t, acc);
                         xcur += TILE * ES;
                         if (to_load > 0) {
-                            load_tile<B, GPT>(buf[i], wl, pl, lane);
-                            wl += d.tile_bytes; pl += d.tile_bytes;
+                            load_tile<B, GPT>(buf[i], wl + i * TB, pl + i * TB, lane);
                             --to_load;
                         }
                     }
                 });
+                wl += NBUF * TB; pl += NBUF * TB;
             }
             // fold the slice in true units: lane (g, t) holds rows g, g+8 x tokens 2t, 2t+1
 #pragma unroll
