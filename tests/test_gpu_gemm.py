@@ -171,3 +171,24 @@ def test_a8_gemm_token_tiles_and_split_k(M, G):
     assert cq.cq_gemm_status(ws) == 0
     assert torch.equal(y1.view(torch.int16), y2.view(torch.int16))
     assert np.array_equal(y_to_numpy(y1), y)
+
+
+def test_random_shapes_both_modes():
+    # seeded shape fuzz: ragged N and K, every width and group size, M on both sides of every dispatch
+    # boundary (16 | 17, token tiles, split-K on / off), a few reserved codes in every case
+    rng = np.random.default_rng(20240607)
+    Ms = [1, 2, 5, 8, 9, 16, 17, 31, 33, 64, 65, 127, 130, 257, 600]
+    for trial in range(28):
+        B = int(rng.integers(1, 9))
+        G = int(rng.choice([32, 64, 128, 256, 512]))
+        K = G * int(rng.integers(1, max(2, 2304 // G)))
+        N = int(rng.integers(1, 420))
+        M = int(rng.choice(Ms))
+        mode = int(rng.integers(0, 2))
+        c = logical_case(N, K, B, G, seed=300 + trial)
+        if B > 1:
+            c.k[int(rng.integers(0, N)), int(rng.integers(0, K))] = -(1 << (B - 1))
+            c = Case(c.k, c.s, c.a, c.b, B, G)
+        x = datagen.activations(M, K, seed=400 + trial, outlier_cols=0.01 if trial % 3 == 0 else 0.0)
+        y, ref = run_both(c, x, mode)
+        check_y(y, ref, f"fuzz trial={trial} B={B} G={G} N={N} K={K} M={M} mode={mode}")
