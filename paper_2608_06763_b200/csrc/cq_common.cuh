@@ -156,14 +156,20 @@ __device__ __forceinline__ float level_q(int i, int M, float a, float b) {
     return __fmul_rn(t, fmaf(t, fmaf(t, c, b), a));
 }
 
-// INT8 carrier of magnitude index i (Eq. carrier): RNE(127 q), clamped to [0, 127].
-// W1 / W2 have only the normalised levels {0, 1}, which sit on the carrier grid.
+// INT8 carrier (Eq. carrier) at the normalised position t = i / M: RNE(127 q(t)), clamped to [0, 127],
+// by the fp32 sequence c = (1 - a) - b, q = t fma(t, fma(t, c, b), a).
+__device__ __forceinline__ int carrier_at(float t, float a, float b) {
+    const float c = __fsub_rn(__fsub_rn(1.0f, a), b);
+    const float q = __fmul_rn(t, fmaf(t, fmaf(t, c, b), a));
+    const int r = __float2int_rn(__fmul_rn(127.0f, q));
+    return min(max(r, 0), 127);
+}
+// INT8 carrier of magnitude index i; W1 / W2 have only the normalised levels {0, 1}, which sit on the carrier grid.
 __device__ __forceinline__ int carrier_of(int B, int i, float a, float b) {
     if (B == 1) return 127;
     if (B == 2) return i ? 127 : 0;
     const int M = (1 << (B - 1)) - 1;
-    int r = __float2int_rn(__fmul_rn(127.0f, level_q(i, M, a, b)));
-    return min(max(r, 0), 127);
+    return carrier_at(__fdiv_rn((float)i, (float)M), a, b);
 }
 
 }  // namespace cq

@@ -132,8 +132,8 @@ __device__ __forceinline__ void group_model(const TileRegs<B, TILE / G> &r, cons
 // One group of a tile, Dynamic A8: INT8 MMAs into int32 partials P_g, then acc += s * P_g.
 // xl = this lane's operand base (row g of the staged block, byte 8 t); ctab = this warp's table space.
 template <int B, int G, int NT, int GI>
-__device__ __forceinline__ void group_a8(const TileRegs<B, TILE / G> &r, const int8_t *xl, int XS, int8_t *ctab, int g,
-                                         int t, float (&acc)[NT][4]) {
+__device__ __forceinline__ void group_a8(const TileRegs<B, TILE / G> &r, const int8_t *xl, int XS, int8_t *ctab,
+                                         const float *tt, int g, int t, float (&acc)[NT][4]) {
     constexpr int MPG = G / 32;                  // MMAs per group
     constexpr int L = B == 1 ? 1 : (1 << (B - 1));
     constexpr int NE = 1 << B;                   // table entries per row
@@ -146,7 +146,8 @@ __device__ __forceinline__ void group_a8(const TileRegs<B, TILE / G> &r, const i
         const float a_lo = __low2float(ab_lo), b_lo = __high2float(ab_lo);
         const float a_hi = __low2float(ab_hi), b_hi = __high2float(ab_hi);
         for (int i = t; i < L; i += 4) {
-            const int c_lo = carrier_of(B, i, a_lo, b_lo), c_hi = carrier_of(B, i, a_hi, b_hi);
+            const float ti = tt[i];   // i / M, divided once per CTA
+            const int c_lo = carrier_at(ti, a_lo, b_lo), c_hi = carrier_at(ti, a_hi, b_hi);
             ctab[g * NE + L + i] = (int8_t)c_lo;
             ctab[g * NE + L - i] = (int8_t)(-c_lo);
             ctab[(g + 8) * NE + L + i] = (int8_t)c_hi;
@@ -187,7 +188,7 @@ __device__ __forceinline__ void group_a8(const TileRegs<B, TILE / G> &r, const i
 
 template <int B, int G, int NT, int MODE>
 __device__ __forceinline__ void compute_tile(const TileRegs<B, TILE / G> &r, const uint8_t *xl, int XS, int8_t *ctab,
-                                             int g, int t, float (&acc)[NT][4]) {
+                                             const float *tt, int g, int t, float (&acc)[NT][4]) {
     constexpr int GPT = TILE / G;
     static_for<GPT>([&](auto gc) {
         constexpr int GI = decltype(gc)::value;
@@ -196,7 +197,7 @@ __device__ __forceinline__ void compute_tile(const TileRegs<B, TILE / G> &r, con
             if (!fix) group_model<B, G, NT, GI, false>(r, reinterpret_cast<const __half *>(xl), XS, acc);
             else group_model<B, G, NT, GI, true>(r, reinterpret_cast<const __half *>(xl), XS, acc);
         } else {
-            group_a8<B, G, NT, GI>(r, reinterpret_cast<const int8_t *>(xl), XS, ctab, g, t, acc);
+            group_a8<B, G, NT, GI>(r, reinterpret_cast<const int8_t *>(xl), XS, ctab, tt, g, t, acc);
         }
     });
 }
@@ -232,6 +233,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
     __shared__ float s_inv[16];
     __shared__ unsigned s_max[16];
     __shared__ int s_last;
+    __shared__ float s_t[MODE == 1 && B >= 3 ? 128 : 1];   // Dynamic A8: t_i = i / M of the carrier tables
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int VT = d.KT + E;                       // virtual units per row block
@@ -239,6 +241,9 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
     const int64_t v_begin = cut_start(blockIdx.x, V, P), v_end = cut_start((int64_t)blockIdx.x + 1, V, P);
     if (threadIdx.x < 16) { s_max[threadIdx.x] = 0; s_inv[threadIdx.x] = 1.0f; }
     int8_t *ctab = nullptr;
+    if constexpr (MODE == 1 && B >= 3) {   // read after the first barrier of the slice loop
+        if (threadIdx.x < L) s_t[threadIdx.x] = __fdiv_rn((float)threadIdx.x, (float)(L - 1));
+    }
     if constexpr (MODE == 1 && B >= 3) ctab = reinterpret_cast<int8_t *>(smem) + RT * (MAX_SUB * TILE + XS_PAD8) + warp * 16 * (1 << B);
 
     bool first_slice = true;
@@ -379,7 +384,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                 static_for<NBUF>([&](auto ic) {
                     constexpr int i = decltype(ic)::value;
                     if (i < left) {
-                        compute_tile<B, G, NT, MODE>(buf[i], xcur, XS, ctab, g, t, acc);
+                        compute_tile<B, G, NT, MODE>(buf[i], xcur, XS, ctab, s_t, g, t, acc);
                         xcur += TILE * ES;
                         if (to_load > 0) {
                             load_tile<B, GPT>(buf[i], wl + i * TB, pl + i * TB, lane);
