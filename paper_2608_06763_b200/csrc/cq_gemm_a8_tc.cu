@@ -1,14 +1,15 @@
 // Large-M Dynamic-A8 GEMM on tcgen05 (Section 5.4): INT8 activation carriers x INT8 weight
 // carriers -> int32 group partials in TMEM -> fp32 rescale by s_g (and d_x / 127 at the end).
 //
-// CTA = 128 output channels x BN tokens, K walked in 128-wide blocks (one layout tile).
+// CTA = 128 output channels x BN tokens, K (or one split-K slice of it) walked in 128-wide blocks (one layout tile).
 //   warp 0       producer: bulk copy of the raw layout tile, TMA of the x8 tile [BN x 128] (swizzled)
 //   warp 1       TMEM allocation, tcgen05.mma kind::i8 (K = 32 per instruction); every group of
 //                the block accumulates into its own BN columns of one of two TMEM buffers
 //   warps 2..17  work warps, two jobs per K block, interleaved so the tensor core never waits on both:
 //                (a) decode block t: a signed carrier table r(k) per (row, group) (Eq. carrier, the
-//                    fp32 sequence of cq_common.cuh), then one table look-up per weight into the
-//                    K-major swizzled INT8 operand tile;
+//                    fp32 sequence of cq_common.cuh), then the carriers of the block (byte-permute look-ups
+//                    in register tables for B <= 4, one shared-memory look-up per weight otherwise) go
+//                    into the K-major swizzled INT8 operand tile in the operand order of cq_decode.cuh;
 //                (b) drain block t-1: tcgen05.ld of its int32 partials P_g, acc += s_g * P_g in fp32
 //                    registers (Eq. a8-output), which frees that TMEM buffer for block t+1.
 //                At the end y = (d_x / 127) * acc, rounded to bf16.

@@ -15,8 +15,9 @@
 // s_g multiplies the fp32 group reduction, as in the paper's narrow path.  Activations go
 // bf16 -> fp16 with a per-token power-of-two scale so that nothing overflows or loses bits.
 //
-// Dynamic A8 uses the INT8 m16n8k32 MMA on signed carriers looked up in a per-warp table of the
-// group's non-negative carriers (Eq. carrier), int32 group partials, fp32 rescale (Eq. a8-output).
+// Dynamic A8 uses the INT8 m16n8k32 MMA on signed carriers (Eq. carrier) taken from a per-(row, group)
+// table indexed by the stored code -- in registers and read with byte permutes for B <= 4, in shared
+// memory otherwise (a8_row_regs in cq_decode.cuh) -- int32 group partials, fp32 rescale (Eq. a8-output).
 #include <cstdlib>
 
 #include "cq_common.cuh"
