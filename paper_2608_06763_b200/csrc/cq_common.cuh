@@ -84,6 +84,15 @@ __host__ __device__ constexpr int pair_pos(int pw, int p) {
     return pw == 4 ? 4 * n : pw == 2 ? 2 * (2 * n + r) : pw == 1 ? 4 * n + ((2 + 2 * (w & 1) + r) & 3) : 8 * (p & 1);
 }
 
+// inverse: the pair stored in slot q (0 .. 16/pw - 1, position q * pw) of word wi of a plane
+__host__ __device__ constexpr int pair_at(int pw, int wi, int q) {
+    if (pw == 8) return 2 * wi + q;
+    if (pw == 4) return 8 * (wi >> 1) + 2 * q + (wi & 1);
+    if (pw == 2) return 8 * wi + 2 * (q >> 1) + (q & 1);
+    const int c = ((q & 3) - 2) & 3;   // pw == 1: bit 4 n + rho, rho = (2 + 2 (w & 1) + r) & 3
+    return 8 * (2 * wi + (c >> 1)) + 2 * (q >> 2) + (c & 1);
+}
+
 // byte offset of word W (0 .. 2B-1) of lane `lane` inside a row block
 __host__ __device__ inline int word_byte_offset(int B, int W, int lane) {
     const int nfq = (2 * B) / 4;

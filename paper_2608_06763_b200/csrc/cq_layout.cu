@@ -58,8 +58,8 @@ __global__ void repack_codes_kernel(const uint8_t *__restrict__ codes, Dims d, i
     const int pw = plane_width(d.B, pl), bo = plane_bit_offset(d.B, pl);
     const int wi = W - plane_word_base(d.B, pl);
     uint32_t word = 0;
-    for (int pair = 0; pair < 32; ++pair) {
-        if (pair_word(pw, pair) != wi) continue;
+    for (int q = 0; q < 16 / pw; ++q) {
+        const int pair = pair_at(pw, wi, q);
         for (int half = 0; half < 2; ++half) {
             int r, kk;
             weight_of(rb, lane, pair, half, r, kk);
@@ -67,7 +67,7 @@ __global__ void repack_codes_kernel(const uint8_t *__restrict__ codes, Dims d, i
             unsigned u;
             if (n < d.N && k < d.K) u = stored_from_field(d.B, canonical_field(codes + n * row_bytes, k, d.B, row_bytes));
             else u = (d.B == 1) ? 1u : (1u << (d.B - 1));  // padding: code 0 (W1: +1), its scale is 0
-            word |= ((u >> bo) & ((1u << pw) - 1u)) << (pair_pos(pw, pair) + 16 * half);
+            word |= ((u >> bo) & ((1u << pw) - 1u)) << (q * pw + 16 * half);
         }
     }
     uint8_t *dst = layout + (size_t)tile * d.tile_bytes + rb * 256 * d.B + word_byte_offset(d.B, W, lane);
