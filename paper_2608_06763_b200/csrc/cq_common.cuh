@@ -165,6 +165,10 @@ __device__ __forceinline__ float level_q(int i, int M, float a, float b) {
     return __fmul_rn(t, fmaf(t, fmaf(t, c, b), a));
 }
 
+// Row stride (bytes) of a shared-memory carrier table of 2^B entries per row: tables read per code
+// (B >= 5) are padded by one word so that the same entry of different rows falls into different banks.
+__host__ __device__ constexpr int carrier_table_stride(int B) { return (1 << B) + (B >= 5 ? 4 : 0); }
+
 // INT8 carrier (Eq. carrier) at the normalised position t = i / M: RNE(127 q(t)), clamped to [0, 127],
 // by the fp32 sequence c = (1 - a) - b, q = t fma(t, fma(t, c, b), a).
 __device__ __forceinline__ int carrier_at(float t, float a, float b) {

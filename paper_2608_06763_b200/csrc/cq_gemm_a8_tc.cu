@@ -70,7 +70,7 @@ __global__ void __launch_bounds__(A8_THREADS, 1)
 gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
     constexpr int GPT = TILE / G;                 // groups per 128-wide block
     constexpr int MPG = 4 / GPT;                  // K = 32 MMAs per group
-    constexpr int NCODE = 1 << B;                 // table entries (indexed by the stored code u)
+    constexpr int NCODE = carrier_table_stride(B);   // bytes per table row (2^B entries indexed by the stored code u, padded)
     constexpr int Mx = B == 1 ? 1 : (1 << (B - 1)) - 1;
     constexpr int B_STAGE_BYTES = BN * 128;
     constexpr uint32_t ACC_COLS = GPT * BN;       // columns of one accumulator buffer
@@ -368,7 +368,7 @@ cudaError_t launch_a8(const void *layout, const Dims &d, const int8_t *x8, int64
     p.partial = partial; p.counters = counters;
     p.raw_stage_bytes = (d.tile_bytes + 1023) / 1024 * 1024;
     const size_t smem = (size_t)A8_STAGES * (A8_A_STAGE_BYTES + BN * 128) + (size_t)A8_RAW_STAGES * p.raw_stage_bytes +
-                        (size_t)8 * 2 * 16 * (1 << B) + (size_t)A8_SRING * 128 * GPT * 4 + 512 + 256;
+                        (size_t)8 * 2 * 16 * carrier_table_stride(B) + (size_t)A8_SRING * 128 * GPT * 4 + 512 + 256;
     auto kern = gemm_a8_kernel<B, G, BN>;
     static bool attr_done = false;
     if (!attr_done) {

@@ -137,7 +137,7 @@ __device__ __forceinline__ void group_a8(const TileRegs<B, TILE / G> &r, const i
                                          const float *tt, int g, int t, float (&acc)[NT][4]) {
     constexpr int MPG = G / 32;                  // MMAs per group
     constexpr int L = B == 1 ? 1 : (1 << (B - 1));
-    constexpr int NE = 1 << B;                   // table entries per row
+    constexpr int NE = carrier_table_stride(B);   // bytes from one row's table to the next
     const uint2 p_lo = r.prm[0][GI], p_hi = r.prm[1][GI];
     uint4 tab_lo = make_uint4(0, 0, 0, 0), tab_hi = make_uint4(0, 0, 0, 0);
     const int8_t *trow_lo = ctab + g * NE, *trow_hi = ctab + (g + 8) * NE;
@@ -245,7 +245,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
     if constexpr (MODE == 1 && B >= 3) {   // read after the first barrier of the slice loop
         if (threadIdx.x < L) s_t[threadIdx.x] = __fdiv_rn((float)threadIdx.x, (float)(L - 1));
     }
-    if constexpr (MODE == 1 && B >= 3) ctab = reinterpret_cast<int8_t *>(smem) + RT * (MAX_SUB * TILE + XS_PAD8) + warp * 16 * (1 << B);
+    if constexpr (MODE == 1 && B >= 3) ctab = reinterpret_cast<int8_t *>(smem) + RT * (MAX_SUB * TILE + XS_PAD8) + warp * 16 * carrier_table_stride(B);
 
     bool first_slice = true;
     for (int64_t v = v_begin; v < v_end;) {
@@ -495,7 +495,7 @@ cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, con
     if (sub64 > MAX_SUB) sub64 = MAX_SUB;
     const int sub_tiles = (int)sub64;
     const int XS = sub_tiles * TILE + XS_PAD;
-    size_t smem = MODE == 0 ? (size_t)RT * XS * 2 : (size_t)RT * (MAX_SUB * TILE + XS_PAD8) + (B >= 3 ? 8 * 16 * (1 << B) : 0);
+    size_t smem = MODE == 0 ? (size_t)RT * XS * 2 : (size_t)RT * (MAX_SUB * TILE + XS_PAD8) + (B >= 3 ? 8 * 16 * carrier_table_stride(B) : 0);
     auto kern = gemv_kernel<B, G, NT, MODE>;
     static bool attr_done = false;
     if (smem > 48 * 1024 && !attr_done) {
