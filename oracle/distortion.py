@@ -75,6 +75,26 @@ def population_distortion(dist: str, B: int, s: float, a: float, b: float) -> fl
     return 2.0 * total
 
 
+def joint_population_distortion(dist: str, B: int, s: float, z, zt) -> float:
+    """D_B^joint(s,a,b) of Eq. carrier-aware-population-objective for given normalised continuous
+    levels z_i and carrier-grid levels zt_i (every code must own a cell: increasing boundaries):
+    2 sum_i integral over (h_{i-1}, h_i) of [(x - s z_i)^2 + (x - s zt_i)^2] / 2 f(x) dx with the
+    boundaries of Eq. carrier-aware-boundary, expanded in the cell moments of
+    Eq. reference-cell-moments."""
+    M = len(z) - 1
+    h = [0.5 * s * ((z[i + 1] ** 2 + zt[i + 1] ** 2) - (z[i] ** 2 + zt[i] ** 2)) / ((z[i + 1] + zt[i + 1]) - (z[i] + zt[i]))
+         for i in range(M)]
+    assert all(h[i + 1] > h[i] for i in range(M - 1)), "a code owns no cell"
+    total, lo = 0.0, 0.0
+    for i in range(M + 1):
+        hi = h[i] if i < M else math.inf
+        mu0, mu1, mu2 = cell_moments(dist, lo, hi)
+        for lev in (z[i], zt[i]):
+            total += 0.5 * (mu2 - 2.0 * s * lev * mu1 + s * s * lev * lev * mu0)
+        lo = hi
+    return 2.0 * total
+
+
 def best_scale(dist: str, B: int, a: float, b: float, lo: float = 0.05, hi: float = 20.0):
     """min over s of D_B(s, a, b): coarse scan then golden-section refinement."""
     grid = np.geomspace(lo, hi, 400)

@@ -156,3 +156,30 @@ def test_joint_encoder_invariants(B):
     # reporting quantity of Eq. carrier-aware-nrmse is well defined and below the INT8-grid-free bound 1
     nrmse = np.sqrt(tot_j / (2.0 * float(np.sum(W.astype(np.float64) ** 2))))
     assert 0 < nrmse < 1
+
+
+@pytest.mark.parametrize("dist", ["gaussian", "laplace", "uniform"])
+@pytest.mark.parametrize("B", [3, 4])
+def test_joint_population_distortion_against_monte_carlo(dist, B):
+    # Eq. carrier-aware-population-objective from closed-form cell moments and the joint boundaries, against
+    # the empirical (L_C + L_A8) / (2 n) of the oracle's joint assignment on unit-variance samples
+    from oracle import distortion
+    a16, b16 = np.float16(0.6), np.float16(-0.25)
+    z, zt = oracle.joint_levels(B, a16, b16)
+    s = {3: 2.2, 4: 2.9}[B] if dist != "uniform" else 1.7
+    want = distortion.joint_population_distortion(dist, B, s, list(z), list(zt))
+    g = datagen.stream(77, f"mc-{dist}-{B}")
+    n = 400_000
+    x = {"gaussian": datagen.normal, "laplace": lambda gg, m: datagen.laplace(gg, m, 1.0 / np.sqrt(2.0)),
+         "uniform": lambda gg, m: datagen.uniform_pm(gg, m, np.sqrt(3.0))}[dist](g, n).astype(np.float32)
+    assert abs(float(np.var(x.astype(np.float64))) - 1.0) < 0.02          # the reference sources have unit variance
+    k = oracle.assign_group_joint(x, B, np.float32(s), a16, b16)
+    lc, la = oracle.group_losses(x, B, np.float32(s), a16, b16, k)
+    got = (lc + la) / (2.0 * n)
+    i = np.abs(k.astype(np.int64))
+    per = 0.5 * ((np.abs(x.astype(np.float64)) - s * z[i]) ** 2 + (np.abs(x.astype(np.float64)) - s * zt[i]) ** 2)
+    se = float(per.std(ddof=1) / np.sqrt(n))
+    assert abs(got - want) <= 5.0 * se + 1e-6, (got, want, se)
+    # and it differs from the continuous distortion at the same parameters whenever the projection moves a level
+    cont = distortion.population_distortion(dist, B, s, float(a16), float(b16))
+    assert want >= cont - 1e-12
