@@ -489,7 +489,6 @@ cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, con
                        const float *dxs, uint16_t *y, int M, int P, int max_run, int E, float *partial, int *counters,
                        cudaStream_t st) {
     constexpr int RT = 8 * NT;
-    constexpr int L = B == 1 ? 1 : (1 << (B - 1));
     int64_t sub64 = max_run;   // the longest run bounds the activation slice a CTA stages
     if (sub64 > d.KT) sub64 = d.KT;
     if (sub64 > MAX_SUB) sub64 = MAX_SUB;
