@@ -187,13 +187,78 @@ __device__ __forceinline__ void group_a8(const TileRegs<B, TILE / G> &r, const i
     }
 }
 
+// One group of a tile, model dtype, W3: with only eight stored codes the group's levels are kept as a
+// signed fp16 table per row -- q(1/3) and q(2/3) by the fp32 Horner form of Eq. gpu-horner, the other
+// entries are 0 and +-1 (u = 0, the reserved pattern, reads 0) -- split into a low-byte and a high-byte
+// register pair.  A half-word of four codes (the selector assembled from the 2-bit and the 1-bit plane,
+// as in a8_row_regs) fetches four levels with two byte permutes, two more interleave the bytes into
+// half2 MMA operands.  K order inside a 32-wide block is the operand order of cq_decode.cuh, which
+// the staged activations follow: k = 16 a + 4 t + 2 h + e at half position 8 t + 4 e + 2 a + h.
+template <int G, int NT, int GI>
+__device__ __forceinline__ void group_model_w3(const TileRegs<3, TILE / G> &r, const __half *xl, int XS, float (&acc)[NT][4]) {
+    constexpr int MPG = G / 32;   // 32-wide k blocks per group, two k = 16 MMAs each
+    uint32_t tlo[2][2], thi[2][2];
+    float sc[2];
+#pragma unroll
+    for (int rr = 0; rr < 2; ++rr) {
+        const uint2 p = r.prm[rr][GI];
+        sc[rr] = __uint_as_float(p.x & 0x7FFFFFFFu);
+        const __half2 ab = as_h2(p.y);
+        const float a = __low2float(ab), b = __high2float(ab), c = (1.0f - a) - b;
+        constexpr float t1 = 1.0f / 3.0f, t2 = 2.0f / 3.0f;
+        const float q1 = t1 * fmaf(t1, fmaf(t1, c, b), a), q2 = t2 * fmaf(t2, fmaf(t2, c, b), a);
+        const uint32_t q12 = as_u32(__floats2half2_rn(q1, q2)), nq = q12 | 0x80008000u;
+        constexpr uint32_t K = 0x003CBC00u;            // bytes 4..7 of a permute: 0x00, 0xBC (-1), 0x3C (+1), 0x00
+        tlo[rr][0] = prmt(q12, 0u, 0x0244u);           // low bytes of  0, -1, -q2, -q1
+        tlo[rr][1] = prmt(q12, 0u, 0x4204u);           //               0, q1, q2, 1
+        thi[rr][0] = prmt(nq, K, 0x1354u);             // high bytes of 0, -1, -q2, -q1
+        thi[rr][1] = prmt(q12, K, 0x6314u);            //               0, q1, q2, 1
+    }
+    float D[NT][4];
+    static_for<MPG>([&](auto mc) {
+        constexpr int mi = decltype(mc)::value, MI = GI * MPG + mi;
+        uint32_t A[2][4];   // [e][a0 a1 a2 a3]
+        static_for<2>([&](auto rc) {
+            constexpr int RR = decltype(rc)::value;
+            constexpr int rho = (2 + 2 * (MI & 1) + RR) & 3;   // where the 1-bit plane keeps this selector's bits
+            const uint32_t x0 = RR ? (r.w[MI] >> 2) : r.w[MI];
+            const uint32_t w1 = r.w[4 + (MI >> 1)];
+            const uint32_t y = rho == 2 ? w1 : rho == 3 ? (w1 >> 1) : rho == 0 ? (w1 << 2) : (w1 << 1);
+            const uint32_t sel = (x0 & 0x33333333u) | (y & 0x44444444u);
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const uint32_t se = e ? (sel >> 16) : sel;
+                const uint32_t lo4 = prmt(tlo[RR][0], tlo[RR][1], se), hi4 = prmt(thi[RR][0], thi[RR][1], se);
+                A[e][RR] = prmt(lo4, hi4, 0x5140u);        // levels of n = 0, 1
+                A[e][2 + RR] = prmt(lo4, hi4, 0x7362u);    // levels of n = 2, 3
+            }
+        });
+#pragma unroll
+        for (int tb = 0; tb < NT; ++tb) {
+            const uint4 bf = *reinterpret_cast<const uint4 *>(xl + tb * 8 * XS + 32 * MI);
+            if constexpr (mi == 0) mma_f16_z(D[tb], A[0], bf.x, bf.y);
+            else mma_f16(D[tb], A[0], bf.x, bf.y);
+            mma_f16(D[tb], A[1], bf.z, bf.w);
+        }
+    });
+#pragma unroll
+    for (int tb = 0; tb < NT; ++tb) {
+        acc[tb][0] = fmaf(sc[0], D[tb][0], acc[tb][0]);
+        acc[tb][1] = fmaf(sc[0], D[tb][1], acc[tb][1]);
+        acc[tb][2] = fmaf(sc[1], D[tb][2], acc[tb][2]);
+        acc[tb][3] = fmaf(sc[1], D[tb][3], acc[tb][3]);
+    }
+}
+
 template <int B, int G, int NT, int MODE>
 __device__ __forceinline__ void compute_tile(const TileRegs<B, TILE / G> &r, const uint8_t *xl, int XS, int8_t *ctab,
                                              const float *tt, int g, int t, float (&acc)[NT][4]) {
     constexpr int GPT = TILE / G;
     static_for<GPT>([&](auto gc) {
         constexpr int GI = decltype(gc)::value;
-        if constexpr (MODE == 0) {
+        if constexpr (MODE == 0 && B == 3) {
+            group_model_w3<G, NT, GI>(r, reinterpret_cast<const __half *>(xl), XS, acc);
+        } else if constexpr (MODE == 0) {
             const bool fix = B > 1 && __any_sync(0xffffffffu, (r.prm[0][GI].x | r.prm[1][GI].x) >> 31);
             if (!fix) group_model<B, G, NT, GI, false>(r, reinterpret_cast<const __half *>(xl), XS, acc);
             else group_model<B, G, NT, GI, true>(r, reinterpret_cast<const __half *>(xl), XS, acc);
@@ -229,7 +294,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
     constexpr int NBUF = (B <= 4) ? 3 : 2;
     constexpr int ES = MODE == 0 ? 2 : 1;  // bytes per staged activation element
     constexpr int CB = 2048 * B, TB = CB + 1024 * GPT;   // bytes of a tile's code part and of a whole tile
-    constexpr int XPAD = MODE == 0 ? XS_PAD : XS_PAD8;
+    constexpr int XPAD = MODE == 0 ? (B == 3 ? 2 * XS_PAD : XS_PAD) : XS_PAD8;   // W3 reads 16 bytes per lane: rows 64 bytes apart in the banks
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ float s_inv[16];
     __shared__ unsigned s_max[16];
@@ -333,15 +398,30 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                     sh = max(min(sh, 100), -100);
                     const float sc = __uint_as_float((uint32_t)(127 + sh) << 23);   // 2^sh
                     if (threadIdx.x == m) s_inv[m] = __uint_as_float((uint32_t)(127 - sh) << 23);
+                    uint32_t ws[4] = {0u, 0u, 0u, 0u};
                     if (c < cpr) {
-                        uint4 v = *(uint4 *)(xs + m * XS + c * 8);
-                        uint32_t ws[4] = {v.x, v.y, v.z, v.w};
+                        const uint4 v = *(const uint4 *)(xs + m * XS + c * 8);
+                        ws[0] = v.x; ws[1] = v.y; ws[2] = v.z; ws[3] = v.w;
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
                             const float lo = __uint_as_float(ws[q] << 16) * sc, hi = __uint_as_float(ws[q] & 0xFFFF0000u) * sc;
                             ws[q] = as_u32(__floats2half2_rn(lo, hi));
                         }
-                        *(uint4 *)(xs + m * XS + c * 8) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
+                    }
+                    if constexpr (B != 3) {
+                        if (c < cpr) *(uint4 *)(xs + m * XS + c * 8) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
+                    } else {
+                        // W3 reads its activations in the operand order of cq_decode.cuh: the four chunks of a
+                        // 32-wide block (four neighbouring lanes) are all read before any of them is rewritten
+                        __syncwarp();
+                        if (c < cpr) {
+                            __half *blk = xs + m * XS + (c >> 2) * 32 + 16 * (c & 1) + 2 * ((c >> 1) & 1);   // t = 2 (c & 1), a = (c >> 1) & 1
+#pragma unroll
+                            for (int tt = 0; tt < 2; ++tt) {   // values k+0, k+2 (e = 0) | k+1, k+3 (e = 1) of t = 2 (c & 1) + tt
+                                *reinterpret_cast<uint32_t *>(blk + 8 * tt) = prmt(ws[2 * tt], ws[2 * tt + 1], 0x5410u);
+                                *reinterpret_cast<uint32_t *>(blk + 8 * tt + 4) = prmt(ws[2 * tt], ws[2 * tt + 1], 0x7632u);
+                            }
+                        }
                     }
                 };
                 if (M <= 2) {   // the common decode case: short plain loops
@@ -379,7 +459,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
             for (int tb = 0; tb < NT; ++tb)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) acc[tb][i] = 0.0f;
-            const uint8_t *xcur = smem + (size_t)(g * XS + (MODE == 0 ? 4 : 8) * t) * ES;  // this lane's B-fragment base, current tile
+            const uint8_t *xcur = smem + (size_t)(g * XS + ((MODE == 0 && B != 3) ? 4 : 8) * t) * ES;  // this lane's B-fragment base, current tile
             int to_load = (ke - ks) - NBUF;                              // tiles not yet requested
             for (int left = ke - ks; left > 0; left -= NBUF) {
                 static_for<NBUF>([&](auto ic) {
@@ -493,7 +573,7 @@ cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, con
     if (sub64 > d.KT) sub64 = d.KT;
     if (sub64 > MAX_SUB) sub64 = MAX_SUB;
     const int sub_tiles = (int)sub64;
-    const int XS = sub_tiles * TILE + XS_PAD;
+    const int XS = sub_tiles * TILE + (B == 3 ? 2 * XS_PAD : XS_PAD);
     size_t smem = MODE == 0 ? (size_t)RT * XS * 2 : (size_t)RT * (MAX_SUB * TILE + XS_PAD8) + (B >= 3 ? 8 * 16 * carrier_table_stride(B) : 0);
     auto kern = gemv_kernel<B, G, NT, MODE>;
     static bool attr_done = false;
