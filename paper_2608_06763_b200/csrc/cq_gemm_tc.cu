@@ -59,6 +59,44 @@ __device__ __forceinline__ uint32_t weight_pair_bf16(const uint32_t (&w)[2 * B],
     return *reinterpret_cast<const uint32_t *>(&v);
 }
 
+// W3: the eight stored codes of a (row, group) index a signed bf16 table of s * sign(k) * q(|k| / 3)
+// (u = 0, the reserved pattern, and k = 0 read zero), kept as a low-byte and a high-byte register pair
+// and read four codes at a time with byte permutes; q(1/3) and q(2/3) by the fp32 Horner form.
+struct W3Table { uint32_t lo[2], hi[2]; };
+__device__ __forceinline__ W3Table w3_table(uint2 p) {
+    const float s = __uint_as_float(p.x & 0x7FFFFFFFu);
+    const __half2 ab = as_h2(p.y);
+    const float a = __low2float(ab), b = __high2float(ab), c = (1.0f - a) - b;
+    constexpr float t1 = 1.0f / 3.0f, t2 = 2.0f / 3.0f;
+    const float q1 = t1 * fmaf(t1, fmaf(t1, c, b), a), q2 = t2 * fmaf(t2, fmaf(t2, c, b), a);
+    const __nv_bfloat162 v12 = __floats2bfloat162_rn(s * q1, s * q2), vs = __floats2bfloat162_rn(s, 0.0f);
+    const uint32_t q12 = *reinterpret_cast<const uint32_t *>(&v12), ss = *reinterpret_cast<const uint32_t *>(&vs);
+    const uint32_t nq = q12 | 0x80008000u, ns = ss | 0x00008000u;
+    W3Table t;                                  // entries u = 0 .. 7:  0, -s, -s q2, -s q1 | 0, s q1, s q2, s
+    t.lo[0] = prmt(nq, ns, 0x0247u) & 0xFFFFFF00u;   // low bytes:  0, (-s).lo, (-s q2).lo, (-s q1).lo
+    t.lo[1] = prmt(q12, ss, 0x4207u) & 0xFFFFFF00u;  //             0, (s q1).lo, (s q2).lo, s.lo
+    t.hi[0] = prmt(nq, ns, 0x1357u) & 0xFFFFFF00u;   // high bytes: 0, (-s).hi, (-s q2).hi, (-s q1).hi
+    t.hi[1] = prmt(q12, ss, 0x5317u) & 0xFFFFFF00u;  //             0, (s q1).hi, (s q2).hi, s.hi
+    return t;
+}
+// the eight weights of row half RR in the 32-wide k block MI, as bf16 pairs in natural k order:
+// out[0] = (k+0, k+1), out[1] = (k+2, k+3) of chunk 2 MI, out[2], out[3] the same of chunk 2 MI + 1
+template <int RR, int MI>
+__device__ __forceinline__ void w3_block(const uint32_t (&w)[6], const W3Table &t, uint32_t (&out)[4]) {
+    constexpr int rho = (2 + 2 * (MI & 1) + RR) & 3;   // where the 1-bit plane keeps this selector's bits
+    const uint32_t x0 = RR ? (w[MI] >> 2) : w[MI];
+    const uint32_t w1 = w[4 + (MI >> 1)];
+    const uint32_t y = rho == 2 ? w1 : rho == 3 ? (w1 >> 1) : rho == 0 ? (w1 << 2) : (w1 << 1);
+    const uint32_t sel = (x0 & 0x33333333u) | (y & 0x44444444u), sel1 = sel >> 16;
+    // selector nibble n = 2 a + h of half-word e holds k = 16 a + 4 t + 2 h + e
+    const uint32_t l0 = prmt(t.lo[0], t.lo[1], sel), h0 = prmt(t.hi[0], t.hi[1], sel);
+    const uint32_t l1 = prmt(t.lo[0], t.lo[1], sel1), h1 = prmt(t.hi[0], t.hi[1], sel1);
+    const uint32_t e0a = prmt(l0, h0, 0x5140u), e0b = prmt(l0, h0, 0x7362u);   // (k+0, k+2) of chunks 2 MI, 2 MI + 1
+    const uint32_t e1a = prmt(l1, h1, 0x5140u), e1b = prmt(l1, h1, 0x7362u);   // (k+1, k+3)
+    out[0] = prmt(e0a, e1a, 0x5410u); out[1] = prmt(e0a, e1a, 0x7632u);
+    out[2] = prmt(e0b, e1b, 0x5410u); out[3] = prmt(e0b, e1b, 0x7632u);
+}
+
 struct TcParams {
     const uint8_t *layout;
     uint16_t *y;
@@ -191,6 +229,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                 }
             }
             const uint8_t *prow = raw + d.code_bytes + ((rb * 16 + g) * GPT) * 8;
+            W3Table w3_lo{}, w3_hi{};   // W3: level tables of rows g and g + 8; one per tile when the group spans it
+            if constexpr (B == 3 && G == 128) {
+                w3_lo = w3_table(*(const uint2 *)prow);
+                w3_hi = w3_table(*(const uint2 *)(prow + 8 * GPT * 8));
+            }
 #pragma unroll 1
             for (int half_k = 0; half_k < 2 && ok; ++half_k) {
                 const int kb = 2 * tile + half_k, s = kb % STAGES;
@@ -204,6 +247,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                     constexpr int JQ = decltype(jq)::value;        // pair of chunks 2 JQ, 2 JQ + 1 of the tile
                     constexpr int gi = (32 * JQ) / G;              // both chunks lie in this group
                     const uint2 p_lo = *(const uint2 *)(prow + gi * 8), p_hi = *(const uint2 *)(prow + (8 * GPT + gi) * 8);
+                    if constexpr (B == 3) {
+                        // table decode (w3_block): no per-weight arithmetic, the reserved pattern reads zero
+                        if constexpr (G < 128) { w3_lo = w3_table(p_lo); w3_hi = w3_table(p_hi); }
+                        uint32_t o_lo[4], o_hi[4];
+                        w3_block<0, JQ>(w, w3_lo, o_lo);
+                        w3_block<1, JQ>(w, w3_hi, o_hi);
+                        static_for<2>([&](auto jc) {
+                            constexpr int jcv = decltype(jc)::value, jl = (2 * JQ + jcv) & 3;
+                            const int off = (((2 * jl + (t >> 1)) ^ g) * 16) + (t & 1) * 8;
+                            *(uint2 *)(row_lo + off) = make_uint2(o_lo[2 * jcv], o_lo[2 * jcv + 1]);
+                            *(uint2 *)(row_hi + off) = make_uint2(o_hi[2 * jcv], o_hi[2 * jcv + 1]);
+                        });
+                        return;
+                    }
                     const RowCoef c_lo = make_coef<B>(p_lo), c_hi = make_coef<B>(p_hi);
                     const bool fix = B > 1 && __any_sync(0xffffffffu, (p_lo.x | p_hi.x) >> 31);  // reserved pattern present
                     auto emit = [&](auto fx) {
