@@ -18,7 +18,7 @@ Workspace plan_workspace(const Dims &d, int64_t M, int mode) {
     Workspace w{};
     const int64_t Kp = (int64_t)d.KT * TILE;
     const int64_t Mc = M < 16 ? M : 16;  // rows handled by one small-M launch
-    const GemvPlan gp = gemv_plan(d, Mc);
+    const GemvPlan gp = gemv_plan(d, Mc, mode);
     size_t off = 0;
     w.status_off = off; off += 256;  // first, so cq_gemm_status finds it without knowing the problem
     // arrival counters: one per 128-row block (small M) or per output tile (split-K GEMM)

@@ -71,6 +71,75 @@ __device__ __forceinline__ __half2 pair_T(const uint32_t (&w)[2 * B]) {
     }
 }
 
+// The small-M kernel's variant, arranged so that every instruction carries at most one literal: a
+// logic or a packed-half instruction encodes a single immediate (and a packed-half FMA none in its
+// addend), so any further constant costs a register move per use unless it lives in a register; the
+// few that must are read once per kernel from constant memory (`DecodeRegs`), which keeps the
+// compiler from folding them back into literals.  What comes out is the signed code in "code units":
+//   B = 1:     +-1, the bit sent straight to the fp16 sign: 0xBC00 ^ (bit << 15)  (a shift and one logic op)
+//   B = 2..6:  the integer k itself: the field is read as base + u under exponent bits chosen by
+//              where the field sits (base = 2^(10 - pos)), and one add of the literal -(base + 2^(B-1))
+//              leaves k, exactly;
+//   B = 7, 8:  T = k / 2^(B-1) by one FMA (scale as the literal, offset from a register): k^3 would
+//              leave the fp16 range.
+// code_unit<B>() is the normalised position t of one unit: t = |T| code_unit.
+template <int B>
+__host__ __device__ constexpr float code_unit() {
+    return B <= 2 ? 1.0f : B <= 6 ? 1.0f / (float)((1 << (B - 1)) - 1) : (float)(1 << (B - 1)) / (float)((1 << (B - 1)) - 1);
+}
+struct DecodeRegs { uint32_t one_neg; uint32_t off; uint32_t magic[4]; };
+__constant__ uint32_t c_decode_consts[8] = {
+    0xBC00BC00u,                                          // -1, -1
+    0xC880C880u,                                          // -9, -9 = -(1024 + 128) / 128, the FMA addend of B = 8
+    0x64006400u, 0x5C005C00u, 0x54005400u, 0x4C004C00u,   // exponent bits for a field at bit 0 / 2 / 4 / 6: base 1024 / 256 / 64 / 16
+    0u, 0u};
+__device__ __forceinline__ DecodeRegs load_decode_regs() {
+    DecodeRegs r;
+    r.one_neg = c_decode_consts[0];
+    r.off = c_decode_consts[1];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) r.magic[i] = c_decode_consts[2 + i];
+    return r;
+}
+__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t c) {   // (a & b) | c
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t lop3_and_xor(uint32_t a, uint32_t b, uint32_t c) {  // (a & b) ^ c
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+template <int B, int P>
+__device__ __forceinline__ __half2 pair_K(const uint32_t (&w)[2 * B], const DecodeRegs &dr) {
+    if constexpr (B == 1) {
+        constexpr int W = pair_word(1, P), pos0 = pair_pos(1, P);
+        const uint32_t word = pos0 == 15 ? w[W] : (w[W] << (15 - pos0));
+        return as_h2(lop3_and_xor(word, 0x80008000u, dr.one_neg));
+    } else if constexpr (B == 2 || B == 4) {
+        constexpr int W = pair_word(B, P), pos0 = pair_pos(B, P);
+        constexpr int shr = pos0 >= 8 ? 8 : 0, pos = pos0 - shr;
+        const uint32_t word = shr ? (w[W] >> shr) : w[W];
+        constexpr uint32_t m = (((1u << B) - 1u) << pos) * 0x00010001u;
+        const uint32_t hbits = lop3_and_or(word, m, dr.magic[pos / 2]);     // base + u, base = 2^(10 - pos)
+        constexpr uint32_t off = half_neg_pow2_plus(10 - pos, B == 2 ? 2 : 8);   // -(base + 2^(B-1))
+        return __hadd2(as_h2(hbits), as_h2(h2dup(off)));
+    } else if constexpr (B == 8) {
+        constexpr int W = pair_word(8, P), pos0 = pair_pos(8, P);
+        const uint32_t word = pos0 ? (w[W] >> 8) : w[W];
+        const uint32_t hbits = lop3_and_or(word, 0x00FF00FFu, dr.magic[0]);
+        return __hfma2(as_h2(hbits), as_h2(h2dup(half_pow2(-7))), as_h2(dr.off));   // (1024 + u) / 128 - 9
+    } else if constexpr (B == 7) {
+        const uint32_t hbits = pair_codes<7, P>(w) | 0x64006400u;
+        // (1024 + u) / 64 - 17 has no register constant of its own: -17 = 2 * (-9) + 1 is not worth a second one
+        return __hfma2(as_h2(hbits), as_h2(h2dup(half_pow2(-6))), as_h2(h2dup(half_neg_pow2_plus(4, 1))));
+    } else {   // B = 3, 5, 6: planes assembled, then the same add
+        const uint32_t hbits = pair_codes<B, P>(w) | 0x64006400u;
+        return __hadd2(as_h2(hbits), as_h2(h2dup(half_neg_pow2_plus(10, 1 << (B - 1)))));
+    }
+}
+
 struct RowCoef { __half2 a2, b2, c2; float s; };
 
 // Coefficients of q as a polynomial in T = k / 2^(B-1):  t = |T| rho, rho = 2^(B-1) / M, so

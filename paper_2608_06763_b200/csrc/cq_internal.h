@@ -30,10 +30,13 @@ struct Workspace {
 };
 Workspace plan_workspace(const Dims &d, int64_t M, int mode);
 
+// Streaming multiprocessors of the current device (148 when no device can be asked).
+int sm_count();
+
 // Decomposition of the small-M path: number of CTAs (one contiguous run of tiles each) and the
 // largest number of CTAs that contribute to one 128-row block.
 struct GemvPlan { int ctas, max_run, overhead; };
-GemvPlan gemv_plan(const Dims &d, int64_t M);
+GemvPlan gemv_plan(const Dims &d, int64_t M, int mode);
 
 // Small-M (M <= 16) split-K tensor-core GEMV, both activation modes.
 cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,

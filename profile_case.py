@@ -1,6 +1,6 @@
 """Run a few launches of one cq_gemm case (for ncu captures and quick timing).
 
-    python -m paper_2608_06763_b200.profile_case --B 4 --G 128 --N 8192 --K 8192 --M 1 --mode 0 --launches 12
+    python profile_case.py --B 4 --G 128 --N 8192 --K 8192 --M 1 --mode 0 --launches 12
 
 Weights rotate over enough copies that no launch finds them in L2.  Prints the CUDA-event time per
 launch.  Inputs are the seeded synthetic tensors the benchmark uses.
@@ -12,7 +12,7 @@ import sys
 import numpy as np
 import torch
 
-sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
 import datagen  # noqa: E402
 import paper_2608_06763_b200 as cq  # noqa: E402
 
