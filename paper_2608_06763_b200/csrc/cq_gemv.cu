@@ -59,10 +59,18 @@ __host__ __device__ constexpr int gemv_x_bytes_max(int B, int NT, int MODE) {
                      : gemv_rows(NT, MODE) * (MAX_SUB * TILE + 2 * XS_PAD) * 2;
 }
 __host__ __device__ constexpr int gemv_smem_budget(int ctas) { return (227 * 1024) / ctas - 2048; }   // dynamic shared memory of a CTA
+// How a CTA's tiles reach the registers.  Straight from global memory into a two- or three-deep register
+// prefetch where that fits the registers (it measured a little faster there); through a shared-memory ring
+// filled by bulk copies where it does not: G = 32 (four parameter records per tile row), the widths made of
+// several bit planes, and the two-token variant.
+__host__ __device__ constexpr bool gemv_uses_ring(int B, int G, int NT, int MODE) {
+    return G == 32 || (B >= 5 && B <= 7) || (MODE == 2 && NT == 2);
+}
 // Resident CTAs per SM: three where the registers (80 per thread: one token block) and a ring of at least
 // four stages allow it, otherwise two.
 __host__ __device__ constexpr int gemv_occ(int B, int G, int NT, int MODE) {
     if (MODE != 2 && NT == 2) return 2;
+    if (!gemv_uses_ring(B, G, NT, MODE)) return CQ_GEMV_CTAS_PER_SM;
     const int tb = 2048 * B + 1024 * (TILE / G);
     return (gemv_smem_budget(CQ_GEMV_CTAS_PER_SM) - (gemv_x_bytes_max(B, NT, MODE) + 127) / 128 * 128) / tb >= 4 ? CQ_GEMV_CTAS_PER_SM : 2;
 }
@@ -107,6 +115,34 @@ struct TileRegs {
     uint2 prm[2][GPT];  // {s bits, a | b << 16} of rows g and g + 8
 };
 
+__device__ __forceinline__ uint4 ld_stream16(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint2 ld_stream8(const void *p) {
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+template <int B, int GPT, class T>
+__device__ __forceinline__ void load_tile_g(T &r, const uint8_t *wl, const uint8_t *pl, int lane) {
+    constexpr int NFQ = (2 * B) / 4;
+#pragma unroll
+    for (int q = 0; q < NFQ; ++q) {
+        const uint4 v = ld_stream16(wl + q * 512);
+        r.w[4 * q + 0] = v.x; r.w[4 * q + 1] = v.y; r.w[4 * q + 2] = v.z; r.w[4 * q + 3] = v.w;
+    }
+    if constexpr ((2 * B) % 4 != 0) {
+        const uint2 v = ld_stream8(wl + NFQ * 512 - lane * 8);
+        r.w[4 * NFQ + 0] = v.x; r.w[4 * NFQ + 1] = v.y;
+    }
+#pragma unroll
+    for (int gi = 0; gi < GPT; ++gi) {
+        r.prm[0][gi] = ld_stream8(pl + gi * 8);
+        r.prm[1][gi] = ld_stream8(pl + (8 * GPT + gi) * 8);
+    }
+}
 // A warp's slice of a ring stage -> registers.  wl = stage + row-block base + lane * 16 (codes);
 // pl = parameter record of row g of the row block.
 template <int B, int GPT>
@@ -463,6 +499,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
             float *__restrict__ partial, int *__restrict__ counters, int nstage, uint32_t ring_off, int *__restrict__ status) {
     constexpr int GPT = TILE / G;
     constexpr int L = B == 1 ? 1 : (1 << (B - 1));
+    constexpr bool RING = gemv_uses_ring(B, G, NT, MODE);
     constexpr bool F16 = MODE != 1;        // activations staged as fp16 (model dtype) or as the INT8 carrier
     constexpr int ES = F16 ? 2 : 1;        // bytes per staged activation element
     constexpr int CB = 2048 * B, TB = CB + 1024 * GPT;   // bytes of a tile's code part and of a whole tile
@@ -518,7 +555,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
         }
         src += (size_t)(first < 0 ? 0 : first) * (size_t)TB;
     }
-    if (warp == 0 && lane < n_tiles && lane < nstage) {
+    if (RING && warp == 0 && lane < n_tiles && lane < nstage) {
         tc::mbar_arrive_expect_tx(&s_full[lane], (uint32_t)TB);
         tc::bulk_load(ring + (size_t)lane * TB, src + (size_t)lane * TB, (uint32_t)TB, &s_full[lane]);
     }
@@ -557,6 +594,25 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                 asm volatile("griddepcontrol.wait;" ::: "memory");
                 asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
                 first_slice = false;
+            }
+            // direct variant: the first tiles of the slice are requested before the activations are staged
+            constexpr int NBUF = RING ? 1 : (B <= 4 ? 3 : 2);
+            const uint8_t *tile0 = layout + ((size_t)nb * d.KT + ks) * (size_t)TB;
+            const uint8_t *wl = tile0 + warp * 256 * B + lane * 16;              // next tile to load (codes)
+            const uint8_t *pl = tile0 + CB + ((warp * 16 + g) * GPT) * 8;        // next tile to load (params)
+            TileRegs<B, GPT> buf0, buf1, buf2;   // separate objects (an array of them ends up in local memory)
+            auto buf_at = [&](auto ic) -> TileRegs<B, GPT> & {
+                constexpr int i = decltype(ic)::value;
+                if constexpr (i == 0) return buf0;
+                else if constexpr (i == 1) return buf1;
+                else return buf2;
+            };
+            if constexpr (!RING) {
+                static_for<NBUF>([&](auto ic) {
+                    constexpr int i = decltype(ic)::value;
+                    if (ks + i < ke) load_tile_g<B, GPT>(buf_at(ic), wl + i * TB, pl + i * TB, lane);
+                });
+                wl += NBUF * TB; pl += NBUF * TB;   // tile offsets inside a round of NBUF loads are immediates
             }
             compute_barrier();  // previous slice fully consumed
 
@@ -670,6 +726,20 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
             for (int tb = 0; tb < NT; ++tb)
                 xo[tb] = (MODE == 2 ? min(tb, M - 1) : min(tb * 8 + g, M - 1)) * XS + ((F16 && B != 3) ? 4 : 8) * t;
             const uint8_t *xcur = smem;
+            if constexpr (!RING) {
+                int to_load = (ke - ks) - NBUF;                              // tiles not yet requested
+                for (int left = ke - ks; left > 0; left -= NBUF) {
+                    static_for<NBUF>([&](auto ic) {
+                        constexpr int i = decltype(ic)::value;
+                        if (i < left) {
+                            compute_tile<B, G, NT, MODE>(buf_at(ic), dr, xcur, xo, ctab, s_t, g, t, acc);
+                            xcur += TILE * ES;
+                            if (to_load > 0) { load_tile_g<B, GPT>(buf_at(ic), wl + i * TB, pl + i * TB, lane); --to_load; }
+                        }
+                    });
+                    wl += NBUF * TB; pl += NBUF * TB;
+                }
+            } else {
 #pragma unroll 1
             for (int kb = ks; kb < ke; ++kb) {
                 // Refill the stage every warp has copied out of by now (that of the previous tile) with the tile
@@ -689,6 +759,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                 if (++st == nstage) { st = 0; ph ^= 1u; }
                 compute_tile<B, G, NT, MODE>(regs, dr, xcur, xo, ctab, s_t, g, t, acc);
                 xcur += TILE * ES;
+            }
             }
             // fold the slice in true units: lane (g, t) holds rows g, g+8 x tokens 2t, 2t+1 (MODE 2: token tb)
 #pragma unroll
@@ -821,10 +892,13 @@ cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, con
     size_t xbytes = MODE != 1 ? (size_t)M * XS * 2 : (size_t)M * (MAX_SUB * TILE + XS_PAD8) + (B >= 3 ? 8 * 16 * carrier_table_stride(B) : 0);
     const uint32_t ring_off = (uint32_t)((xbytes + 127) / 128 * 128);
     constexpr int OCC = gemv_occ(B, G, NT, MODE);
-    int nstage = (int)((gemv_smem_budget(OCC) - (int64_t)ring_off) / TB);
-    if (nstage > MAX_STAGES) nstage = MAX_STAGES;
-    if (nstage > max_run) nstage = max_run < 2 ? 2 : max_run;   // a run never holds more tiles than this
-    if (nstage < 2) return cudaErrorInvalidConfiguration;
+    int nstage = 0;
+    if (gemv_uses_ring(B, G, NT, MODE)) {
+        nstage = (int)((gemv_smem_budget(OCC) - (int64_t)ring_off) / TB);
+        if (nstage > MAX_STAGES) nstage = MAX_STAGES;
+        if (nstage > max_run) nstage = max_run < 2 ? 2 : max_run;   // a run never holds more tiles than this
+        if (nstage < 2) return cudaErrorInvalidConfiguration;
+    }
     const size_t smem = ring_off + (size_t)nstage * TB;
     auto kern = gemv_kernel<B, G, NT, MODE>;
     static std::atomic<uint64_t> attr_done{0};
