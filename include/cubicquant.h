@@ -123,8 +123,9 @@ int cq_gemm_host(const void *layout, int B, int G, const uint16_t *x_host, uint1
  *   - CQ_ERR_WORKSPACE when the problem needs more scratch than the built-in array holds
  *     (cq_workspace_bytes(B, G, M, N, K, CQ_MODEL_DTYPE) > CQ_STATIC_SCRATCH_BYTES);
  *     CQ_ERR_UNSUPPORTED for M > 16 or an unsupported format.
- *   - The first call on each device looks up the array's device address (with that device current).
- *     Make that first call during start-up, before any stream capture begins.
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     where the CUDA runtime loads modules lazily, that is also the moment the array's memory is
+ *     committed on that device.  Make that first call during start-up, before any stream capture begins.
  *   - Every call on a device shares the one array and finds in it what the previous call left; the
  *     call clears the counters it relies on before launching.  Two calls whose kernels may overlap
  *     on the GPU (different streams, or host threads) race on the array: serialise them. */
@@ -148,6 +149,14 @@ int cq_decode_weights(const void *layout, int B, int G, int64_t N, int64_t K, fl
 /* Integer group partials of Eq. a8-output: P[M][N][K/G] int32 from x8[M][K]. */
 int cq_debug_a8_partials(const void *layout, int B, int G, const int8_t *x8, int64_t M, int64_t N, int64_t K,
                          int32_t *P, void *stream);
+
+/* The bounded device-side wait on its own (the pipelined kernels give every wait on a barrier a limit;
+ * the paper has no counterpart, it is this library's failure reporting).  Launches one thread that
+ * waits on a barrier nobody arrives on, with nothing in flight, gives up after `limit_cycles` SM clock
+ * cycles (1 .. 2e9) and records that in the workspace's status word; the kernel then ends normally.
+ * Afterwards cq_gemm_status(workspace) returns CQ_ERR_TIMEOUT until the workspace is re-initialised.
+ * workspace: device pointer, 16-byte aligned, at least 512 bytes. */
+int cq_debug_wait_timeout(void *workspace, size_t workspace_bytes, int64_t limit_cycles, void *stream);
 
 /* ---- Offline encoder (the step before the hot path; Sections 4.1 and 4.3) --------------------------
  * W[N][K] float, logical signed codes k[N][K] int8 (what cq_pack_codes takes), scale[N][K/G] float,

@@ -59,6 +59,8 @@ def lib():
         L.cq_decode_carriers.argtypes = [vp, i, i, i64, i64, vp, vp]
         L.cq_decode_weights.argtypes = [vp, i, i, i64, i64, vp, vp]
         L.cq_debug_a8_partials.argtypes = [vp, i, i, vp, i64, i64, i64, vp, vp]
+        L.cq_debug_wait_timeout.argtypes = [vp, sz, i64, vp]
+        L.cq_debug_wait_timeout.restype = i
         L.cq_encode_assign.argtypes = [vp, i, i, i64, i64, vp, vp, vp, i, vp, vp]
         L.cq_encode_scale.argtypes = [vp, vp, i, i, i64, i64, vp, vp, i, vp, vp]
         L.cq_encode_losses.argtypes = [vp, vp, i, i, i64, i64, vp, vp, vp, vp, vp, vp]
@@ -230,6 +232,12 @@ def cq_debug_a8_partials(pw: PackedWeights, x8: torch.Tensor) -> torch.Tensor:
     _check(lib().cq_debug_a8_partials(_ptr(pw.layout), pw.B, pw.G, _ptr(x8), M, pw.N, pw.K, _ptr(out), _stream()),
            "cq_debug_a8_partials")
     return out
+
+
+def cq_debug_wait_timeout(workspace: torch.Tensor, limit_cycles: int = 2_000_000):
+    """One bounded wait that runs out (about a millisecond by default); the workspace's status word records it."""
+    _check(lib().cq_debug_wait_timeout(_ptr(workspace), workspace.numel() * workspace.element_size(), limit_cycles,
+                                       _stream()), "cq_debug_wait_timeout")
 
 
 CQ_FIT_CONTINUOUS, CQ_FIT_JOINT = 0, 1

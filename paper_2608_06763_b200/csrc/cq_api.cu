@@ -9,6 +9,7 @@
 namespace cq {
 
 static thread_local int g_last_cuda_error = 0;
+void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = (int)e; }
 
 int gemm_tc_available();
 
@@ -249,6 +250,15 @@ int cq_decode_weights(const void *layout, int B, int G, int64_t N, int64_t K, fl
     if (!What) return CQ_ERR_INVALID_ARG;
     CQ_DEBUG_PROLOGUE();
     return wrap(launch_decode_weights(layout, d, What, (cudaStream_t)stream));
+}
+
+int cq_debug_wait_timeout(void *workspace, size_t workspace_bytes, int64_t limit_cycles, void *stream) {
+    if (!workspace || workspace_bytes < 512 || limit_cycles <= 0 || limit_cycles > 2000000000ll) return CQ_ERR_INVALID_ARG;
+    if (misaligned(workspace)) return CQ_ERR_ALIGNMENT;
+    const int st = check_arch();
+    if (st != CQ_OK) return st;
+    // the status word is the first word of every workspace (plan_workspace)
+    return wrap(launch_wait_timeout((int *)workspace, (long long)limit_cycles, (cudaStream_t)stream));
 }
 
 int cq_debug_a8_partials(const void *layout, int B, int G, const int8_t *x8, int64_t M, int64_t N, int64_t K,

@@ -450,11 +450,8 @@ cudaError_t launch_encode_losses(const float *W, const int8_t *k, int B, int G, 
 cudaError_t launch_encode_search(const float *W, int B, int G, int64_t N, int64_t K, int joint, int effort, int8_t *k,
                                  float *scale, uint16_t *a, uint16_t *b, cudaStream_t st) {
     const int64_t groups = N * (K / G);
-    static bool attr_done = false;
-    if (!attr_done) {   // the per-thread work arrays live in local memory: prefer L1 over shared memory
-        cudaFuncSetAttribute(search_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 0);
-        attr_done = true;
-    }
+    static std::atomic<uint64_t> attr_done{0};   // the per-thread work arrays live in local memory: prefer L1 over shared memory
+    (void)ensure_func_attr(search_kernel, attr_done, cudaFuncAttributePreferredSharedMemoryCarveout, 0);
     search_kernel<<<(unsigned)((groups + 31) / 32), 32, 0, st>>>(W, B, G, N, K, joint, effort, k, scale, a, b);
     return cudaGetLastError();
 }

@@ -32,7 +32,7 @@ int gemm_a8_split_k(const Dims &d, int64_t M) {
     const int64_t bnt = gemm_a8_token_tile(d, M);
     const int64_t ctas = (int64_t)d.NB * ((M + bnt - 1) / bnt);
     if (ctas >= 100 || M > 256) return 1;
-    int64_t sk = 148 / ctas;
+    int64_t sk = sm_count() / ctas;
     if (sk > 8) sk = 8;
     if (sk > d.KT / 4) sk = d.KT / 4;   // at least four layout tiles per slice
     return sk < 1 ? 1 : (int)sk;
@@ -166,14 +166,22 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
         float acc[QCOLS];
 #pragma unroll
         for (int i = 0; i < QCOLS; ++i) acc[i] = 0.0f;
+        // A wait that gives up (bounded, see mbar_wait) must not make this warp leave the loop: with G = 128
+        // its partner of the row block would then wait for it at the 64-thread barrier for ever.  The warp
+        // keeps walking the blocks instead, without waiting any more, so every barrier still sees both
+        // warps; what it computes from then on is discarded (the status word is set, nothing is stored).
         bool ok = true;
-        for (int t = 0; t <= KT && ok; ++t) {
+        auto wait_or_give_up = [&](uint64_t *bar, uint32_t parity, int code) {
+            if (!ok) return;
+            const bool flipped = mbar_wait(bar, parity, prm.status, code);
+            ok = !__any_sync(0xffffffffu, !flipped);   // the warp decides as one
+        };
+        for (int t = 0; t <= KT; ++t) {
             if (t < KT) {
                 // ---------------- (a) decode block t
                 const int rs = t % A8_RAW_STAGES, s = t % A8_STAGES;
-                ok = mbar_wait(&raw_full[rs], (t / A8_RAW_STAGES) & 1, prm.status, 16);
-                if (ok && t >= A8_STAGES) ok = mbar_wait(&st_empty[s], ((t / A8_STAGES) - 1) & 1, prm.status, 17);
-                if (!ok) break;
+                wait_or_give_up(&raw_full[rs], (t / A8_RAW_STAGES) & 1, 16);
+                if (t >= A8_STAGES) wait_or_give_up(&st_empty[s], ((t / A8_STAGES) - 1) & 1, 17);
                 const uint8_t *raw = sRaw + rs * prm.raw_stage_bytes;
                 const uint8_t *rbp = raw + rb * 256 * B;
                 uint32_t w[2 * B];
@@ -266,8 +274,7 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
             if (t >= 1) {
                 // ---------------- (b) drain block t - 1
                 const int td = t - 1, ab = td & 1;
-                ok = mbar_wait(&acc_full[ab], (td >> 1) & 1, prm.status, 18);
-                if (!ok) break;
+                wait_or_give_up(&acc_full[ab], (td >> 1) & 1, 18);
                 tc_fence_after();
                 const float *scd = sScale + (size_t)(td % A8_SRING) * 128 * GPT + drow * GPT;
 #pragma unroll
@@ -370,12 +377,9 @@ cudaError_t launch_a8(const void *layout, const Dims &d, const int8_t *x8, int64
     const size_t smem = (size_t)A8_STAGES * (A8_A_STAGE_BYTES + BN * 128) + (size_t)A8_RAW_STAGES * p.raw_stage_bytes +
                         (size_t)8 * 2 * 16 * carrier_table_stride(B) + (size_t)A8_SRING * 128 * GPT * 4 + 512 + 256;
     auto kern = gemm_a8_kernel<B, G, BN>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    static std::atomic<uint64_t> attr_done{0};   // per kernel instantiation: the devices it has been set on
+    cudaError_t ea = ensure_func_attr(kern, attr_done, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (ea != cudaSuccess) return ea;
     dim3 grid((unsigned)d.NB, (unsigned)((M + BN - 1) / BN), (unsigned)gemm_a8_split_k(d, M));
     kern<<<grid, A8_THREADS, smem, st>>>(xmap, p);
     return cudaGetLastError();

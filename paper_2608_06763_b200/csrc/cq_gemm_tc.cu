@@ -31,7 +31,7 @@ int gemm_tc_split_k(const Dims &d, int64_t M) {
     const int64_t bnt = gemm_tc_token_tile(M);
     const int64_t ctas = (int64_t)d.NB * ((M + bnt - 1) / bnt);
     if (ctas >= 100 || M > 256) return 1;   // the combine of a large token tile costs more than the idle SMs
-    int64_t sk = 148 / ctas;
+    int64_t sk = sm_count() / ctas;
     if (sk > 8) sk = 8;
     if (sk > d.KT / 4) sk = d.KT / 4;   // at least four layout tiles per slice
     return sk < 1 ? 1 : (int)sk;
@@ -396,12 +396,9 @@ cudaError_t launch_bn(const void *layout, const Dims &d, const uint16_t *x, uint
     p.raw_stage_bytes = (d.tile_bytes + 1023) / 1024 * 1024;
     const size_t smem = (size_t)STAGES * (A_STAGE_BYTES + NACC * BN * 128) + (size_t)RAW_STAGES * p.raw_stage_bytes + 256;
     auto kern = gemm_tc_kernel<B, G, BN, NACC>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    static std::atomic<uint64_t> attr_done{0};   // per kernel instantiation: the devices it has been set on
+    cudaError_t ea = ensure_func_attr(kern, attr_done, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (ea != cudaSuccess) return ea;
     p.partial = partial; p.counters = counters;
     dim3 grid((unsigned)d.NB, (unsigned)((M + BN * NACC - 1) / (BN * NACC)), (unsigned)gemm_tc_split_k(d, M));
     kern<<<grid, TC_THREADS, smem, st>>>(xmap, p);

@@ -30,7 +30,6 @@
 // Dynamic A8 uses the INT8 m16n8k32 MMA on signed carriers (Eq. carrier) taken from a per-(row, group)
 // table indexed by the stored code -- in registers and read with byte permutes for B <= 4, in shared
 // memory otherwise (a8_row_regs in cq_decode.cuh) -- int32 group partials, fp32 rescale (Eq. a8-output).
-#include <atomic>
 #include <cstdlib>
 
 #include "cq_common.cuh"
@@ -865,19 +864,6 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
     }
 }
 
-// cudaFuncSetAttribute is a per-device setting: remember, per kernel instantiation, the devices it was made on.
-template <class Kern>
-cudaError_t ensure_smem_attr(Kern kern, std::atomic<uint64_t> &done, int bytes) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    const uint64_t bit = 1ull << (dev & 63);
-    if (dev < 64 && (done.load(std::memory_order_acquire) & bit)) return cudaSuccess;
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess && dev < 64) done.fetch_or(bit, std::memory_order_release);
-    return e;
-}
-
 template <int B, int G, int NT, int MODE>
 cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, const int8_t *xq, int64_t x8_pitch,
                        const float *dxs, uint16_t *y, int M, int P, int max_run, int E, float *partial, int *counters,
@@ -902,7 +888,7 @@ cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, con
     const size_t smem = ring_off + (size_t)nstage * TB;
     auto kern = gemv_kernel<B, G, NT, MODE>;
     static std::atomic<uint64_t> attr_done{0};
-    cudaError_t e = ensure_smem_attr(kern, attr_done, gemv_smem_budget(OCC));
+    cudaError_t e = ensure_func_attr(kern, attr_done, cudaFuncAttributeMaxDynamicSharedMemorySize, gemv_smem_budget(OCC));
     if (e != cudaSuccess) return e;
     // Programmatic dependent launch: this kernel may begin (and prefetch weights) while the previous
     // kernel of the stream drains; it waits for that kernel before touching anything but the weights.

@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "cq_common.cuh"
 
 namespace cq {
@@ -19,6 +21,8 @@ cudaError_t launch_a8_partials(const void *layout, const Dims &d, const int8_t *
 cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, int64_t x8_pitch, float *dx,
                                bool operand_order, cudaStream_t st);
 
+cudaError_t launch_wait_timeout(int *status, long long limit_cycles, cudaStream_t st);
+
 // Workspace carving (all offsets 256-byte aligned).
 struct Workspace {
     size_t counters_off, counters_bytes;   // int32 arrival counters, one per 128-row block
@@ -32,6 +36,24 @@ Workspace plan_workspace(const Dims &d, int64_t M, int mode);
 
 // Streaming multiprocessors of the current device (148 when no device can be asked).
 int sm_count();
+
+// cudaFuncSetAttribute is a per-DEVICE setting: `done` (one per kernel instantiation) remembers, as a bit
+// mask, the devices on which it has been made, so a process that uses several GPUs sets it on each.
+// Thread safe; devices beyond 63 simply set the attribute on every launch.
+template <class Kern>
+cudaError_t ensure_func_attr(Kern kern, std::atomic<uint64_t> &done, cudaFuncAttribute attr, int value) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const bool tracked = dev >= 0 && dev < 64;
+    const uint64_t bit = tracked ? (1ull << dev) : 0;
+    if (tracked && (done.load(std::memory_order_acquire) & bit)) return cudaSuccess;
+    e = cudaFuncSetAttribute(kern, attr, value);
+    if (e == cudaSuccess && tracked) done.fetch_or(bit, std::memory_order_release);
+    return e;
+}
+// the thread's record of the last failed CUDA call (what cq_last_cuda_error returns)
+void set_last_cuda_error(cudaError_t e);
 
 // Decomposition of the small-M path: number of CTAs (one contiguous run of tiles each) and the
 // largest number of CTAs that contribute to one 128-row block.

@@ -2,6 +2,7 @@
 // quantiser.  All of them are one-time or test-side operations except cq::launch_quantize_a8.
 #include "cq_common.cuh"
 #include "cq_internal.h"
+#include "cq_tc_ptx.cuh"
 
 namespace cq {
 
@@ -371,6 +372,23 @@ cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *
     if (M > 64 && threads > 256) threads = 256;    // many rows: smaller CTAs fill the SMs better
     if (operand_order) quantize_a8_kernel<true><<<(unsigned)M, (unsigned)threads, 0, st>>>(x, M, K, x8, x8_pitch, dx);
     else quantize_a8_kernel<false><<<(unsigned)M, (unsigned)threads, 0, st>>>(x, M, K, x8, x8_pitch, dx);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- cq_debug_wait_timeout
+// The bounded wait of the pipelined kernels, on its own: one thread waits on a barrier that nobody
+// arrives on (nothing is in flight, nothing is copied), gives up after `limit` cycles and records the
+// code in the status word, exactly as a stuck pipeline stage would.  The kernel then returns normally.
+__global__ void wait_timeout_kernel(int *status, long long limit) {
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x == 0) {
+        tc::mbar_init(&bar, 1);
+        tc::fence_barrier_init();
+        (void)tc::mbar_wait(&bar, 0, status, 99, limit);
+    }
+}
+cudaError_t launch_wait_timeout(int *status, long long limit_cycles, cudaStream_t st) {
+    wait_timeout_kernel<<<1, 32, 0, st>>>(status, limit_cycles);
     return cudaGetLastError();
 }
 

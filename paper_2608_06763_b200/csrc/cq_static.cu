@@ -7,6 +7,8 @@
 
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "cq_common.cuh"
 #include "cq_internal.h"
 
@@ -20,7 +22,14 @@ constexpr int MAX_DEVICES = 64;
 static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
 
 // device address of g_static_scratch on each device, filled in by the first call on that device
-unsigned char *g_scratch_ptr[MAX_DEVICES] = {};
+// (atomic: host threads may make their first calls at the same time; they all store the same address)
+std::atomic<unsigned char *> g_scratch_ptr[MAX_DEVICES];
+
+// a failed CUDA call: remember its code for cq_last_cuda_error() and report CQ_ERR_CUDA
+int cuda_failed(cudaError_t e) {
+    cq::set_last_cuda_error(e);
+    return CQ_ERR_CUDA;
+}
 
 }  // namespace
 
@@ -36,21 +45,28 @@ extern "C" int cq_gemv_static(const void *layout, int B, int G, const uint16_t *
     if (plan.total > STATIC_SCRATCH_BYTES) return CQ_ERR_WORKSPACE;  // problem too large for the built-in scratch
 
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return CQ_ERR_CUDA;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_failed(e);
     if (dev < 0 || dev >= MAX_DEVICES) return CQ_ERR_UNSUPPORTED;
     int major = 0;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return CQ_ERR_CUDA;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_failed(e);
     if (major != 10) return CQ_ERR_ARCH;
-    if (!g_scratch_ptr[dev]) {
+    unsigned char *ws = g_scratch_ptr[dev].load(std::memory_order_acquire);
+    if (!ws) {
         // one-time set-up for this device (it is the current device): resolve the array's device address
-        unsigned char *p = nullptr;
-        if (cudaGetSymbolAddress((void **)&p, g_static_scratch) != cudaSuccess || !p) return CQ_ERR_CUDA;
-        g_scratch_ptr[dev] = p;
+        e = cudaGetSymbolAddress((void **)&ws, g_static_scratch);
+        if (e != cudaSuccess) return cuda_failed(e);
+        if (!ws) return cuda_failed(cudaErrorInvalidSymbol);
+        g_scratch_ptr[dev].store(ws, std::memory_order_release);
     }
-    unsigned char *ws = g_scratch_ptr[dev];
     cudaStream_t st = (cudaStream_t)stream;
-    // the array keeps whatever the previous call left: the arrival counters must start at zero
-    if (cudaMemsetAsync(ws + plan.counters_off, 0, plan.counters_bytes, st) != cudaSuccess) return CQ_ERR_CUDA;
-    return launch_gemv(layout, d, x, y, M, CQ_MODEL_DTYPE, ws, plan, st) == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+    // the array keeps whatever the previous call left: the arrival counters and the status word must start at zero
+    e = cudaMemsetAsync(ws + plan.status_off, 0, 256, st);
+    if (e != cudaSuccess) return cuda_failed(e);
+    e = cudaMemsetAsync(ws + plan.counters_off, 0, plan.counters_bytes, st);
+    if (e != cudaSuccess) return cuda_failed(e);
+    e = launch_gemv(layout, d, x, y, M, CQ_MODEL_DTYPE, ws, plan, st);
+    return e == cudaSuccess ? CQ_OK : cuda_failed(e);
 }
 #pragma GCC visibility pop

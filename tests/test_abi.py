@@ -56,4 +56,9 @@ def test_argument_errors_are_found_before_any_launch():
     assert L.cq_gemm(one, 4, 128, one, one, 1, 128, 128, 0, one, 16, None) == -4        # workspace too small
     assert L.cq_repack(None, one, one, one, 4, 128, 128, 128, one, None) == -1
     assert L.cq_quantize_a8(one, 0, 128, one, one, None) == -1
+    assert L.cq_debug_wait_timeout(None, 512, 1000, None) == -1
+    assert L.cq_debug_wait_timeout(one, 512, 0, None) == -1               # limit outside 1 .. 2e9
+    assert L.cq_debug_wait_timeout(one, 512, 3 * 10 ** 9, None) == -1
+    assert L.cq_debug_wait_timeout(one, 64, 1000, None) == -1             # too small to hold the status word
+    assert L.cq_debug_wait_timeout(odd, 512, 1000, None) == -3
     assert cq.cq_status_string(-4) == "CQ_ERR_WORKSPACE"

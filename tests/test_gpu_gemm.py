@@ -192,3 +192,22 @@ def test_random_shapes_both_modes():
         x = datagen.activations(M, K, seed=400 + trial, outlier_cols=0.01 if trial % 3 == 0 else 0.0)
         y, ref = run_both(c, x, mode)
         check_y(y, ref, f"fuzz trial={trial} B={B} G={G} N={N} K={K} M={M} mode={mode}")
+
+
+def test_bounded_wait_gives_up_and_is_reported():
+    # the failure path of the pipelined kernels without any failure: one wait on a barrier nobody arrives
+    # on, with nothing in flight, runs out after about a millisecond; the kernel ends normally, the status
+    # word says CQ_ERR_TIMEOUT, and the same workspace serves a correct product once it is re-initialised
+    c = logical_case(256, 512, 4, 128, seed=700)
+    x = x_to_device(datagen.activations(40, 512, seed=701))
+    ws = torch.zeros(cq.cq_workspace_bytes(4, 128, 40, 256, 512, 0), dtype=torch.uint8, device="cuda")
+    assert cq.cq_gemm_status(ws) == 0
+    cq.cq_debug_wait_timeout(ws, 2_000_000)
+    assert cq.cq_gemm_status(ws) == -7 and cq.cq_status_string(-7) == "CQ_ERR_TIMEOUT"
+    assert cq.cq_gemm_status(ws) == -7            # sticky until the workspace is re-initialised
+    cq.cq_workspace_init(ws)
+    assert cq.cq_gemm_status(ws) == 0
+    y = y_to_numpy(cq.cq_gemm(c.pw, x, cq.CQ_MODEL_DTYPE, ws))
+    assert cq.cq_gemm_status(ws) == 0
+    xb = x.view(torch.int16).cpu().numpy().view(np.uint16)
+    check_y(y, oracle.gemm_model(c.codes, c.s, c.a, c.b, 4, 128, 512, xb), "after a reported timeout")

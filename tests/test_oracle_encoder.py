@@ -112,7 +112,7 @@ def test_zero_group_and_zero_weight():
 
 def test_finite_group_table_soft_pin():
     # Section 3.6 table: G128, 15,360 samples, W2..W6, W8.  The paper's random stream is unnamed, so the
-    # pin is the ratio Cubic / clipped INT (<= paper's ratio + 0.015) and exact ties at W2.
+    # pin is the ratio Cubic / clipped INT (<= paper's ratio + 0.01) and exact ties at W2.
     table = {(r[0], int(r[1])): (float(r[2]), float(r[3])) for r in read_table("finite_group_nrmse.txt")}
     n = 15360
     for dist in ("uniform", "gaussian", "laplace"):
@@ -132,7 +132,7 @@ def test_finite_group_table_soft_pin():
             if B == 2:
                 assert abs(res["reference"] - res["int_clipped"]) < 1e-3 * clip
             else:
-                assert res["reference"] / res["int_clipped"] <= cub / clip + 0.015, (dist, B, res, cub, clip)
+                assert res["reference"] / res["int_clipped"] <= cub / clip + 0.01, (dist, B, res, cub, clip)
 
 
 # ----------------------------------------------------------------------------- Dynamic A8

@@ -6,6 +6,7 @@ import math
 import numpy as np
 import pytest
 
+import datagen
 import oracle
 from conftest import read_table
 
@@ -199,3 +200,32 @@ def test_w3_free_codebook_identity():
         from oracle.distortion import normalised_levels
         R = normalised_levels(3, a, b)
         assert abs(R[1] - p1) < 1e-12 and abs(R[2] - p2) < 1e-12 and abs(R[3] - 1) < 1e-12
+
+
+# ----------------------------------------------------------------------------- binary16 conversion
+def test_half_conversion_matches_ieee_binary16():
+    # every fit is serialised through the oracle's own double -> binary16 rounding: pin it to numpy's
+    # float16 (an independent IEEE implementation): exact decode of all 65536 patterns, round trip,
+    # round-to-nearest-even at every midpoint, subnormals, and the overflow threshold
+    L = oracle.lib()
+    bits = np.arange(65536, dtype=np.uint16)
+    want = bits.view(np.float16).astype(np.float64)
+    got = np.array([L.cqo_half_to_double(int(h)) for h in bits])
+    finite = np.isfinite(want)
+    assert np.array_equal(got[finite], want[finite]) and np.all(np.isinf(got[np.isinf(want)])) and np.all(np.isnan(got[np.isnan(want)]))
+    assert np.array_equal(np.signbit(got[finite]), np.signbit(want[finite]))           # -0 keeps its sign
+    back = np.array([L.cqo_double_to_half(float(v)) for v in want[finite]], dtype=np.uint16)
+    assert np.array_equal(back, bits[finite])
+    # midpoints between neighbouring non-negative halves (ties go to the even mantissa), and points just off them
+    pos = want[(bits < 0x7C00)]
+    mids = 0.5 * (pos[:-1] + pos[1:])
+    probes = np.concatenate([mids, np.nextafter(mids, np.inf), np.nextafter(mids, -np.inf), -mids])
+    g = datagen.stream(77, "half-probes")
+    rnd = np.concatenate([datagen.normal(g, 20000), datagen.normal(g, 20000) * 1e-6, datagen.normal(g, 20000) * 3e4,
+                          [65504.0, 65519.999, 65520.0, 65536.0, 1e9, -65520.0, 2.0 ** -24, 2.0 ** -25, 2.0 ** -25 * 1.0000001,
+                           2.0 ** -14, np.nextafter(2.0 ** -14, 0), 0.0, -0.0]])
+    probes = np.concatenate([probes, rnd])
+    with np.errstate(over="ignore"):
+        ref = probes.astype(np.float16).view(np.uint16)
+    mine = np.array([L.cqo_double_to_half(float(v)) for v in probes], dtype=np.uint16)
+    assert np.array_equal(mine, ref), np.flatnonzero(mine != ref)[:10]
