@@ -190,6 +190,33 @@ def logical_quantized_cuda(N: int, K: int, B: int, G: int, seed: int, device="cu
     return k, s, a, b
 
 
+def weights_cuda(kind: str, N: int, K: int, seed: int, device="cuda", **kw):
+    """fp32 weight matrix [N, K] of the same distributions as ``weights`` (normal / laplace / outlier), drawn
+    with torch's seeded generator on the GPU for tensors of 10^8 .. 10^9 entries (the numpy stream takes
+    minutes there).  The stream differs from the numpy one."""
+    import torch
+    gen = torch.Generator(device=device)
+    gen.manual_seed(int(seed) * 2654435761 % (1 << 31) + {"normal": 1, "laplace": 2, "outlier": 3}[kind])
+    W = torch.empty((N, K), dtype=torch.float32, device=device)
+    rows = max(1, (1 << 25) // K)  # slabs bound the temporaries
+    for r0 in range(0, N, rows):
+        r1 = min(N, r0 + rows)
+        shp = (r1 - r0, K)
+        if kind == "normal":
+            W[r0:r1] = torch.randn(shp, generator=gen, device=device) * kw.get("sigma", 0.02)
+        elif kind == "laplace":
+            d = (torch.rand(shp, generator=gen, device=device) - 0.5).clamp(-0.4999999, 0.4999999)
+            W[r0:r1] = -kw.get("b", 0.015) * torch.sign(d) * torch.log1p(-2.0 * d.abs())
+        elif kind == "outlier":
+            base = torch.randn(shp, generator=gen, device=device) * kw.get("sigma", 0.02)
+            sel = torch.rand(shp, generator=gen, device=device) < kw.get("p", 0.001)
+            big = torch.randn(shp, generator=gen, device=device) * kw.get("sigma_out", 0.2)
+            W[r0:r1] = torch.where(sel, big, base)
+        else:
+            raise ValueError(kind)
+    return W
+
+
 def activations_cuda(M: int, K: int, seed: int, outlier_cols: float = 0.0, outlier_scale: float = 20.0, device="cuda"):
     """bf16 N(0,1) activations [M, K] drawn on the GPU (optionally a seeded set of columns scaled)."""
     import torch

@@ -1,10 +1,15 @@
 """Parity at the full sizes of the five benchmark configurations, in the launch configuration the
-benchmark times (same entry point, same dispatch), on outputs the oracle computes one by one:
-whole y where that is cheap, otherwise a seeded sample of activation rows x output channels.
+benchmark times (same entry point, same dispatch, weights produced the same way), on outputs the oracle
+computes one by one: whole y where that is cheap, otherwise a seeded sample of activation rows x output
+channels that always includes the first and last channel / token of the matrix and of a tile.
 
-Weights of configuration 1 are fitted by the oracle encoder; the larger tensors use the seeded
-already-quantised recipe of datagen (running the fitter on 10^8..10^9 weights takes too long), which
-the library packs itself while the oracle packs the sampled rows with its own packer."""
+Weights follow the configurations' recipes: drawn from the stated distribution and fitted by the
+encoder.  Configuration 1 is fitted by the oracle encoder itself; the larger tensors by cq_encode, whose
+output is the oracle encoder's bit for bit (tests/test_gpu_encode.py at small sizes, and re-checked here
+on sampled rows of every full-size tensor).  The 10^8 .. 10^9-entry tensors of configurations 3 - 5 are
+drawn with the seeded GPU generator of datagen.weights_cuda."""
+import functools
+
 import numpy as np
 import pytest
 import torch
@@ -26,6 +31,47 @@ def sampled_reference(k_rows, s_rows, a_rows, b_rows, B, G, K, x_bits, mode, row
     return oracle.gemm_a8(codes, s_rows, a_rows, b_rows, B, G, K, x8, dx, rows=rows)
 
 
+def sample_with_edges(gen, n, count, tile):
+    """`count` seeded indices of range(n) plus the first / last index of the range and of a tile."""
+    idx = gen.choice(n, min(count, n), replace=False)
+    edges = [0, n - 1, tile - 1, tile, n - tile, n // 2]
+    return np.unique(np.concatenate([idx, [e for e in edges if 0 <= e < n]]))
+
+
+class Fitted:
+    """A full-size tensor fitted on the GPU, packed for the library, with host copies of sampled channels."""
+
+    def __init__(self, W, B, G, sample_gen, n_cols):
+        self.B, self.G = B, G
+        self.N, self.K = W.shape
+        k, s, a, b = cq.cq_encode(W, B, G, cq.CQ_FIT_CONTINUOUS, "fast")
+        self.pw = cq.cq_repack(cq.cq_pack_codes(k, B), s, a, b, B, G, self.N, self.K)
+        self.cols = sample_with_edges(sample_gen, self.N, n_cols, 128)
+        ci = torch.from_numpy(self.cols).cuda()
+        self.k, self.s = k[ci].cpu().numpy(), s[ci].cpu().numpy()
+        self.a, self.b = a[ci].cpu().numpy(), b[ci].cpu().numpy()
+        # the encoder on the GPU and the oracle encoder agree on these rows bit for bit
+        probe = self.cols[:: max(1, len(self.cols) // 6)][:6]
+        Wp = W[torch.from_numpy(probe).cuda()].cpu().numpy()
+        ko, so, ao, bo = oracle.encode(Wp, B, G, "fast")
+        sel = np.searchsorted(self.cols, probe)
+        assert np.array_equal(ko, self.k[sel]) and np.array_equal(so, self.s[sel])
+        assert np.array_equal(np.asarray(ao).view(np.uint16), self.a[sel].view(np.uint16))
+        assert np.array_equal(np.asarray(bo).view(np.uint16), self.b[sel].view(np.uint16))
+
+    def check(self, x, mode, what, rows=None):
+        """x: bf16 [M, K] on the device."""
+        M = x.shape[0]
+        ws = torch.zeros(cq.cq_workspace_bytes(self.B, self.G, M, self.N, self.K, mode), dtype=torch.uint8, device="cuda")
+        y = cq.cq_gemm(self.pw, x, mode, ws)
+        assert cq.cq_gemm_status(ws) == 0
+        xb = x.view(torch.int16).cpu().numpy().view(np.uint16)
+        ref = sampled_reference(self.k, self.s, self.a, self.b, self.B, self.G, self.K, xb, mode, rows=rows)
+        ci = torch.from_numpy(self.cols).cuda()
+        got = y[:, ci] if rows is None else y[torch.from_numpy(rows).cuda()][:, ci]
+        check_y(got.float().cpu().numpy().astype(np.float64), ref, what)
+
+
 def test_config1_w4_g128_gemv_oracle_encoded():
     # 4096 x 4096, N(0, 0.02^2) seed 0, fitted by the oracle encoder, x ~ N(0,1), M = 1
     N = K = 4096
@@ -41,73 +87,63 @@ def test_config1_w4_g128_gemv_oracle_encoded():
     assert np.linalg.norm(ref - exact) / np.linalg.norm(exact) < 0.15
 
 
-@pytest.mark.parametrize("B,G", [(1, 32), (2, 128), (3, 64), (4, 128), (6, 32), (8, 128)])
-def test_config2_sweep_cases_full_size(B, G):
-    N = K = 8192
-    k, s, a, b = datagen.logical_quantized(N, K, B, G, seed=1, name=f"sweep-B{B}-G{G}")
-    dk = torch.from_numpy(k).cuda()
-    pw = cq.cq_repack(cq.cq_pack_codes(dk, B), torch.from_numpy(s).cuda(), torch.from_numpy(np.ascontiguousarray(a)).cuda(),
-                      torch.from_numpy(np.ascontiguousarray(b)).cuda(), B, G, N, K)
-    xb = datagen.activations(1, K, seed=1, name="x-sweep")
-    y = y_to_numpy(cq.cq_gemm(pw, x_to_device(xb), cq.CQ_MODEL_DTYPE))
-    ref = oracle.gemm_model(oracle.pack(k, B), s, a, b, B, G, K, xb)
-    check_y(y, ref, f"config 2 B={B} G={G}")
+@functools.lru_cache(maxsize=1)
+def sweep_matrix():
+    # configuration 2: one 8192 x 8192 Laplace(0, 0.015) matrix, seed 1, for every (B, G) of the sweep
+    return torch.from_numpy(datagen.weights("laplace", 8192, 8192, seed=1, b=0.015)).cuda()
 
 
-@pytest.mark.parametrize("name,K,N", [("gate_up", 4096, 28672), ("down", 14336, 4096)])
-@pytest.mark.parametrize("M", [1, 16])
-def test_config3_decode_linears(name, K, N, M):
-    B, G = 4, 128
-    k, s, a, b = datagen.logical_quantized(N, K, B, G, seed=2, name=name)
-    dk = torch.from_numpy(k).cuda()
-    pw = cq.cq_repack(cq.cq_pack_codes(dk, B), torch.from_numpy(s).cuda(), torch.from_numpy(np.ascontiguousarray(a)).cuda(),
-                      torch.from_numpy(np.ascontiguousarray(b)).cuda(), B, G, N, K)
-    xb = datagen.activations(M, K, seed=2)
-    y = y_to_numpy(cq.cq_gemm(pw, x_to_device(xb), cq.CQ_MODEL_DTYPE))
-    cols = np.sort(datagen.stream(2, "cols-" + name).choice(N, 1024, replace=False))
-    ref = sampled_reference(k[cols], s[cols], a[cols], b[cols], B, G, K, xb, cq.CQ_MODEL_DTYPE)
-    check_y(y[:, cols], ref, f"config 3 {name} M={M}")
+@pytest.mark.parametrize("G", [32, 64, 128])
+@pytest.mark.parametrize("B", [1, 2, 3, 4, 6, 8])
+def test_config2_sweep_all_cases_full_size(B, G):
+    f = Fitted(sweep_matrix(), B, G, datagen.stream(1, f"cols-sweep-{B}-{G}"), 1024)
+    x = x_to_device(datagen.activations(1, 8192, seed=1, name="x-sweep"))
+    f.check(x, cq.CQ_MODEL_DTYPE, f"config 2 B={B} G={G}")
 
 
-@pytest.mark.parametrize("mode", [cq.CQ_MODEL_DTYPE, cq.CQ_DYN_A8])
+@functools.lru_cache(maxsize=2)
+def decode_linear(name, seed):
+    # configurations 3 and 4: N(0, 0.02^2) with 0.1 % of the entries replaced by N(0, 0.2^2)
+    K, N = {n: (k, nn) for n, k, nn in datagen.LLAMA8B_SHAPES}[name]
+    return datagen.weights_cuda("outlier", N, K, seed=seed, sigma=0.02, sigma_out=0.2, p=0.001)
+
+
+@pytest.mark.parametrize("name", ["qkv", "o", "gate_up", "down"])
+def test_config3_decode_linears_all_shapes_and_rows(name):
+    W = decode_linear(name, 2)
+    f = Fitted(W, 4, 128, datagen.stream(2, "cols-" + name), 1024)
+    for M in (1, 4, 8, 16):
+        x = x_to_device(datagen.activations(M, W.shape[1], seed=2, name=f"x-{M}"))
+        f.check(x, cq.CQ_MODEL_DTYPE, f"config 3 {name} M={M}")
+
+
 @pytest.mark.parametrize("B", [4, 8])
-def test_config4_crossover_shape_m1024(B, mode):
-    # qkv 4096 -> 6144, activations with 1 % of columns scaled x20, M = 1024
-    K, N, G, M = 4096, 6144, 128, 1024
-    k, s, a, b = datagen.logical_quantized(N, K, B, G, seed=3, name="qkv")
-    dk = torch.from_numpy(k).cuda()
-    pw = cq.cq_repack(cq.cq_pack_codes(dk, B), torch.from_numpy(s).cuda(), torch.from_numpy(np.ascontiguousarray(a)).cuda(),
-                      torch.from_numpy(np.ascontiguousarray(b)).cuda(), B, G, N, K)
-    xb = datagen.activations(M, K, seed=3, outlier_cols=0.01)
-    y = y_to_numpy(cq.cq_gemm(pw, x_to_device(xb), mode))
-    g = datagen.stream(3, "sample")
-    cols = np.sort(g.choice(N, 256, replace=False))
-    rows = np.sort(g.choice(M, 48, replace=False))
-    ref = sampled_reference(k[cols], s[cols], a[cols], b[cols], B, G, K, xb, mode, rows=rows)
-    check_y(y[np.ix_(rows, cols)], ref, f"config 4 B={B} mode={mode}")
+@pytest.mark.parametrize("name", ["qkv", "o", "gate_up", "down"])
+def test_config4_crossover_all_shapes_rows_and_modes(name, B):
+    # same four shapes (seed 3), W4 and W8, M in {1, 16, 64, 256, 1024}, activations with 1 % of the
+    # columns scaled x20, both activation modes
+    W = decode_linear(name, 3)
+    K = W.shape[1]
+    f = Fitted(W, B, 128, datagen.stream(3, f"cols-{name}-{B}"), 256)
+    g = datagen.stream(3, "rows")
+    for M in (1, 16, 64, 256, 1024):
+        x = datagen.activations_cuda(M, K, seed=3 + M, outlier_cols=0.01)
+        rows = None if M <= 64 else sample_with_edges(g, M, 40, 256)
+        for mode in (cq.CQ_MODEL_DTYPE, cq.CQ_DYN_A8):
+            f.check(x, mode, f"config 4 {name} B={B} M={M} mode={mode}", rows=rows)
 
 
 @pytest.mark.parametrize("name,K,N", [("gate_up", 8192, 57344), ("down", 28672, 8192)])
-@pytest.mark.parametrize("B", [3, 4])
-def test_config5_prefill_gemm(name, K, N, B):
-    # M = 4096 tokens, Llama-3-70B MLP shapes, model dtype; drawn on the GPU, sampled rows x channels
-    G, M = 128, 4096
-    k, s, a, b = datagen.logical_quantized_cuda(N, K, B, G, seed=4)
-    pw = cq.cq_repack(cq.cq_pack_codes(k, B), s, a, b, B, G, N, K)
+def test_config5_prefill_gemm_both_modes(name, K, N):
+    # M = 4096 tokens, Llama-3-70B MLP shapes, W ~ N(0, 0.015^2) seed 4, W3 and W4, model dtype and Dynamic A8
+    M = 4096
+    W = datagen.weights_cuda("normal", N, K, seed=4, sigma=0.015)
     x = datagen.activations_cuda(M, K, seed=4)
-    ws = torch.zeros(cq.cq_workspace_bytes(B, G, M, N, K, 0), dtype=torch.uint8, device="cuda")
-    y = cq.cq_gemm(pw, x, cq.CQ_MODEL_DTYPE, ws)
-    assert cq.cq_gemm_status(ws) == 0
     g = datagen.stream(4, "sample-" + name)
-    cols = np.sort(g.choice(N, 256, replace=False))
-    rows = np.sort(g.choice(M, 32, replace=False))
-    # tile edges on purpose: first and last channel / token of the matrix and of a 128 / 512 tile
-    cols[:4] = [0, 127, 128, N - 1]
-    rows[:4] = [0, 511, 512, M - 1]
-    cols, rows = np.unique(cols), np.unique(rows)
-    ci = torch.from_numpy(cols).cuda()
-    xb = x.view(torch.int16).cpu().numpy().view(np.uint16)
-    ref = sampled_reference(k[ci].cpu().numpy(), s[ci].cpu().numpy(), a[ci].cpu().numpy(), b[ci].cpu().numpy(),
-                            B, G, K, xb, cq.CQ_MODEL_DTYPE, rows=rows)
-    got = y[torch.from_numpy(rows).cuda()][:, ci].float().cpu().numpy().astype(np.float64)
-    check_y(got, ref, f"config 5 {name} B={B}")
+    rows = sample_with_edges(g, M, 28, 512)
+    for B in (3, 4):
+        f = Fitted(W, B, 128, g, 200)
+        for mode in (cq.CQ_MODEL_DTYPE, cq.CQ_DYN_A8):
+            f.check(x, mode, f"config 5 {name} B={B} mode={mode}", rows=rows)
+        del f
+        torch.cuda.empty_cache()
