@@ -9,11 +9,13 @@ cq_gemm call per sweep case (18 launches).  Metric: packed-GEMV HBM GB/s = sum o
 effective weight bytes K*N*(B+64/G)/8 divided by the step time.  Every case rotates over enough
 copies of its weights that consecutive launches of a case never find them in L2.
 
-Inputs are seeded synthetic tensors: the sweep's weight matrix is Laplace(0, 0.015) noise encoded by the
-library's own encoder (whose output equals the oracle encoder's), packed and re-tiled by the library's
-kernels; the secondary tables use datagen.logical_quantized_cuda (codes with the bell shape of fitted
-codes, shape parameters in the strictly monotone domain).  Kernels have no value-dependent control flow,
-so throughput does not depend on how the codes were fitted.
+Inputs are seeded synthetic tensors that follow the five benchmark configurations: weights drawn from
+the stated distribution (Laplace / Gaussian / Gaussian with 0.1 % outliers) and fitted by the library's own
+encoder (whose output equals the oracle encoder's), packed and re-tiled by the library's kernels; only the
+table on the paper's own G = 512 measurement shapes uses datagen.logical_quantized_cuda.
+
+--gpus N: N independent replicas of the same job, one process per GPU (the path does not shard).  Under
+torchrun the flag must equal WORLD_SIZE; without torchrun and N > 1 the script relaunches itself under it.
 """
 from __future__ import annotations
 
@@ -34,9 +36,11 @@ SWEEP_B = [1, 2, 3, 4, 6, 8]
 SWEEP_G = [32, 64, 128]
 SWEEP_N = SWEEP_K = 8192
 L2_BYTES = 126 * 1024 * 1024
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the W4 G128 8192x8192 M=1 GEMV, from the
-# ncu capture summarised in profiles/gemv_w4g128_8192_m1.md (algorithmic bytes: 37.78 MB)
-NCU_TRAFFIC_W4G128_BYTES = 37818624
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the W4 G128 8192x8192 M=1 GEMV, from an ncu
+# capture of that kernel (algorithmic bytes: 37.78 MB)
+NCU_TRAFFIC_W4G128_BYTES = 37835520
+# targets the benchmark spec sets for the three kernels, as fractions of the relevant peak
+TARGET_GEMV_FRAC, TARGET_GEMM_FRAC = 0.75, 0.60
 
 
 def eff_bytes(N, K, B, G):
@@ -128,12 +132,27 @@ def build_case(cq, torch, Wd, B, G, copies):
     return pws
 
 
+def fit_pack(cq, W, B, G):
+    """Fit an fp32 matrix on the GPU (fast effort, continuous objective), pack and re-tile it."""
+    N, K = W.shape
+    k, s, a, b = cq.cq_encode(W, B, G, cq.CQ_FIT_CONTINUOUS, "fast")
+    pw = cq.cq_repack(cq.cq_pack_codes(k, B), s, a, b, B, G, N, K)
+    del k
+    return pw
+
+
 def make_packed_cuda(cq, datagen, N, K, B, G, seed):
     k, s, a, b = datagen.logical_quantized_cuda(N, K, B, G, seed)
     codes = cq.cq_pack_codes(k, B)
     pw = cq.cq_repack(codes, s, a, b, B, G, N, K)
     del k, codes
     return pw
+
+
+def rotating(cq, pw, min_copies=2):
+    """Enough copies of a layout that consecutive launches never find it in L2."""
+    n = max(min_copies, int(np.ceil(2 * L2_BYTES / pw.layout.numel())) + 1)
+    return [pw] + [cq.PackedWeights(pw.layout.clone(), pw.B, pw.G, pw.N, pw.K) for _ in range(n - 1)]
 
 
 def time_graph(torch, stream, fn, reps):
@@ -151,19 +170,58 @@ def time_graph(torch, stream, fn, reps):
     return best
 
 
+def int8_peak(torch, stream):
+    """Dense INT8 tensor throughput of this GPU as torch._int_mm (cuBLASLt) reaches it on 8192^3, best of 10:
+    the measured denominator of the Dynamic-A8 roofline (the bf16 one is measured the same way with cuBLAS)."""
+    try:
+        n = 8192
+        a = torch.randint(-127, 128, (n, n), dtype=torch.int8, device="cuda")
+        b = torch.randint(-127, 128, (n, n), dtype=torch.int8, device="cuda").t()
+        torch._int_mm(a, b)
+        best = 1e30
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream); torch._int_mm(a, b); e1.record(stream); stream.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        return {"tops": round(2.0 * n ** 3 / (best * 1e-3) / 1e12, 1), "how": "torch._int_mm 8192^3, best of 10, CUDA events"}
+    except Exception as exc:  # no INT8 GEMM in this torch build: fall back to the nominal figure
+        return {"tops": 4500.0, "how": f"nominal dense INT8 (torch._int_mm unavailable: {type(exc).__name__})"}
+
+
 def extra_suites(torch, cq, datagen, stream, peaks):
-    """Secondary workloads reported beside the headline: prefill-scale GEMM (Llama-3-70B MLP shapes,
-    M = 4096, W3/W4 G128), Llama-3-8B decode linears at M in {1,4,8,16}, and the model-dtype versus
-    Dynamic-A8 crossover in M."""
+    """Secondary workloads reported beside the headline, each on its configuration's recipe: configuration 1
+    (4096^2 W4 G128 M = 1), the prefill GEMM (configuration 5), the Llama-3-8B decode linears (3) and the
+    model-dtype versus Dynamic-A8 crossover in M (4)."""
     out = {}
-    # ---- prefill GEMM
+    hbm = peaks["hbm_gbs"]
+    # ---- configuration 1: W ~ N(0, 0.02^2) seed 0, 4096 x 4096, W4 G128, M = 1
+    W = torch.from_numpy(datagen.weights("normal", 4096, 4096, seed=0, sigma=0.02)).cuda()
+    cp = rotating(cq, fit_pack(cq, W, 4, 128))
+    del W
+    x = torch.from_numpy(datagen.activations(1, 4096, seed=0).view(np.int16)).cuda().view(torch.bfloat16)
+    y = torch.empty((1, 4096), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros(cq.cq_workspace_bytes(4, 128, 1, 4096, 4096, 0), dtype=torch.uint8, device="cuda")
+    fn = lambda i: cq.cq_gemm(cp[i % len(cp)], x, cq.CQ_MODEL_DTYPE, ws, y)
+    fn(0)
+    ms = time_graph(torch, stream, fn, len(cp))
+    b1 = eff_bytes(4096, 4096, 4, 128) + 4 * 4096
+    out["config1_gemv_4096"] = {"us": round(ms * 1e3, 2), "gbs": round(b1 / (ms * 1e-3) / 1e9, 1),
+                                "frac_of_measured_hbm": round(b1 / (ms * 1e-3) / 1e9 / hbm, 4),
+                                "ideal_us_at_measured_hbm": round(b1 / hbm / 1e3, 2)}
+    del cp
+    torch.cuda.empty_cache()
+    # ---- measured INT8 peak
+    i8 = int8_peak(torch, stream)
+    out["int8_peak"] = i8
+    # ---- configuration 5: prefill GEMM, W ~ N(0, 0.015^2) seed 4, W3 / W4 G128, M = 4096, both modes
     gemm = []
     M = 4096
     for name, K, N in datagen.LLAMA70B_MLP_SHAPES:
+        W = datagen.weights_cuda("normal", N, K, seed=4, sigma=0.015)
         x = datagen.activations_cuda(M, K, seed=4)
         y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
         for B in (3, 4):
-            pw = make_packed_cuda(cq, datagen, N, K, B, 128, 4)
+            pw = fit_pack(cq, W, B, 128)
             ws = torch.zeros(cq.cq_workspace_bytes(B, 128, M, N, K, 0), dtype=torch.uint8, device="cuda")
             for _ in range(2):
                 cq.cq_gemm(pw, x, cq.CQ_MODEL_DTYPE, ws, y)
@@ -179,46 +237,61 @@ def extra_suites(torch, cq, datagen, stream, peaks):
             tops = 2.0 * M * N * K / (ms8 * 1e-3) / 1e12
             gemm.append({"shape": name, "K": K, "N": N, "M": M, "B": B, "G": 128, "mode": "dyn_a8",
                          "ms": round(ms8, 4), "tops": round(tops, 1),
+                         "frac_of_measured_int8": round(tops / i8["tops"], 4),
                          "frac_of_nominal_int8_dense_4500": round(tops / 4500.0, 4),
                          "note": "includes the activation quantiser launch"})
             del pw, ws, ws8
-        del x, y
+        del x, y, W
         torch.cuda.empty_cache()
     out["gemm_prefill"] = gemm
-    # ---- decode linears and crossover
-    dec, cross = [], []
+    # ---- configuration 3: decode linears, W ~ N(0, 0.02^2) with 0.1 % N(0, 0.2^2) outliers seed 2, W4 G128,
+    # model dtype, M in {1, 4, 8, 16}, x ~ N(0, 1)
+    dec = []
     for name, K, N in datagen.LLAMA8B_SHAPES:
-        pws = {B: make_packed_cuda(cq, datagen, N, K, B, 128, 2) for B in (4, 8)}
-        copies = {B: [pws[B]] + [cq.PackedWeights(pws[B].layout.clone(), B, 128, N, K)
-                                 for _ in range(int(np.ceil(2 * L2_BYTES / pws[B].layout.numel())))] for B in (4, 8)}
-        for M in (1, 4, 8, 16, 64, 256, 1024):
+        W = datagen.weights_cuda("outlier", N, K, seed=2, sigma=0.02, sigma_out=0.2, p=0.001)
+        cp = rotating(cq, fit_pack(cq, W, 4, 128))
+        del W
+        for M in (1, 4, 8, 16):
+            x = datagen.activations_cuda(M, K, seed=2)
+            y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+            ws = torch.zeros(cq.cq_workspace_bytes(4, 128, M, N, K, 0), dtype=torch.uint8, device="cuda")
+            fn = lambda i: cq.cq_gemm(cp[i % len(cp)], x, cq.CQ_MODEL_DTYPE, ws, y)
+            fn(0)
+            ms = time_graph(torch, stream, fn, max(len(cp), 8))
+            nbytes = eff_bytes(N, K, 4, 128) + 2 * M * (K + N)
+            dec.append({"shape": name, "K": K, "N": N, "M": M, "us": round(ms * 1e3, 2),
+                        "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1), "frac_of_measured_hbm": round(nbytes / (ms * 1e-3) / 1e9 / hbm, 4)})
+        del cp
+        torch.cuda.empty_cache()
+    out["decode_linears_w4g128"] = dec
+    # ---- configuration 4: crossover, the same shapes (seed 3), W4 and W8 G128, M in {1, 16, 64, 256, 1024},
+    # x ~ N(0, 1) with 1 % of the columns scaled x20, both modes
+    cross = []
+    for name, K, N in datagen.LLAMA8B_SHAPES:
+        W = datagen.weights_cuda("outlier", N, K, seed=3, sigma=0.02, sigma_out=0.2, p=0.001)
+        copies = {B: rotating(cq, fit_pack(cq, W, B, 128)) for B in (4, 8)}
+        del W
+        for M in (1, 16, 64, 256, 1024):
             x = datagen.activations_cuda(M, K, seed=3, outlier_cols=0.01)
             y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
             for B in (4, 8):
                 t = {}
                 for mode in (cq.CQ_MODEL_DTYPE, cq.CQ_DYN_A8):
-                    if mode == cq.CQ_DYN_A8 and M not in (1, 16, 64, 256, 1024):
-                        continue
                     ws = torch.zeros(cq.cq_workspace_bytes(B, 128, M, N, K, mode), dtype=torch.uint8, device="cuda")
                     cp = copies[B]
                     fn = lambda i: cq.cq_gemm(cp[i % len(cp)], x, mode, ws, y)
                     fn(0)
                     t[mode] = time_graph(torch, stream, fn, max(len(cp), 8) if M <= 64 else 4)
-                if B == 4 and M <= 16:
-                    dec.append({"shape": name, "K": K, "N": N, "M": M, "us": round(t[0] * 1e3, 2),
-                                "gbs": round(eff_bytes(N, K, 4, 128) / (t[0] * 1e-3) / 1e9, 1)})
-                if 1 in t:
-                    cross.append({"shape": name, "B": B, "M": M, "us_model": round(t[0] * 1e3, 2),
-                                  "us_a8": round(t[1] * 1e3, 2), "model_over_a8": round(t[0] / t[1], 3)})
-        del pws, copies
+                cross.append({"shape": name, "B": B, "M": M, "us_model": round(t[0] * 1e3, 2),
+                              "us_a8": round(t[1] * 1e3, 2), "model_over_a8": round(t[0] / t[1], 3)})
+        del copies
         torch.cuda.empty_cache()
     # ---- the paper's own kernel-measurement shapes (Section 6.3: G512, W2/W5/W8, M in {1,16,64,256}),
     # so B200 numbers can sit beside its H200 table (context only)
     paper = []
     for N, K in ((3584, 3072), (6144, 3584)):
         for B in (2, 5, 8):
-            pw = make_packed_cuda(cq, datagen, N, K, B, 512, 5)
-            cp = [pw] + [cq.PackedWeights(pw.layout.clone(), B, 512, N, K) for _ in range(int(np.ceil(2 * L2_BYTES / pw.layout.numel())))]
+            cp = rotating(cq, make_packed_cuda(cq, datagen, N, K, B, 512, 5))
             for M in (1, 16, 64, 256):
                 x = datagen.activations_cuda(M, K, seed=5)
                 y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
@@ -230,7 +303,7 @@ def extra_suites(torch, cq, datagen, stream, peaks):
                     t[mode] = time_graph(torch, stream, fn, len(cp))
                 paper.append({"N": N, "K": K, "B": B, "G": 512, "M": M, "ms_a16": round(t[0], 5), "ms_a8": round(t[1], 5),
                               "a16_over_a8": round(t[0] / t[1], 3)})
-            del pw, cp
+            del cp
             torch.cuda.empty_cache()
     # ---- offline encoder (the step before the hot path): 4096 x 4096, W4 G128, fast effort, both objectives
     enc = []
@@ -249,7 +322,6 @@ def extra_suites(torch, cq, datagen, stream, peaks):
     del Wd
     out["encoder_gpu"] = enc
     out["paper_h200_shapes_on_b200"] = paper
-    out["decode_linears_w4g128"] = dec
     out["crossover"] = cross
     first = {}
     for c in cross:
@@ -257,6 +329,17 @@ def extra_suites(torch, cq, datagen, stream, peaks):
         if c["model_over_a8"] > 1.0 and key not in first:
             first[key] = c["M"]
     out["crossover_first_M_where_a8_is_faster"] = first
+    # ---- compact summaries of the two tensor-core kernels (W4 G128 gate_up 8192 -> 57344, M = 4096)
+    gm = next(r for r in gemm if r["shape"] == "gate_up" and r["B"] == 4 and r["mode"] == "model_dtype")
+    ga = next(r for r in gemm if r["shape"] == "gate_up" and r["B"] == 4 and r["mode"] == "dyn_a8")
+    out["roofline_gemm"] = {"bound": "tensor", "kernel": "gemm_tc_kernel<B=4,G=128> (tcgen05 kind::f16)", "shape": "M=4096 N=57344 K=8192",
+                            "achieved": gm["tflops"], "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                            "peak_source": peaks["source"] + " (cuBLAS bf16 burst)", "frac": gm["frac_of_measured_bf16_burst"],
+                            "target_frac": TARGET_GEMM_FRAC, "target_met": gm["frac_of_measured_bf16_burst"] >= TARGET_GEMM_FRAC}
+    out["roofline_a8"] = {"bound": "tensor", "kernel": "quantize_a8 + gemm_a8_kernel<B=4,G=128> (tcgen05 kind::i8)",
+                          "shape": "M=4096 N=57344 K=8192", "achieved": ga["tops"], "peak": i8["tops"], "unit": "TOP/s",
+                          "peak_source": "measured: " + i8["how"], "frac": ga["frac_of_measured_int8"],
+                          "target_frac": TARGET_GEMM_FRAC, "target_met": ga["frac_of_measured_int8"] >= TARGET_GEMM_FRAC}
     return out
 
 
@@ -352,7 +435,8 @@ def run_ours(args, rank, world):
         roofline = {"bound": "hbm", "kernel": "gemv_kernel<B=4,G=128,NT=1,model>", "achieved": round(achieved, 1),
                     "peak": peaks["hbm_gbs"], "peak_source": peaks["source"] + " (burst copy)", "unit": "GB/s",
                     "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": NCU_TRAFFIC_W4G128_BYTES,
-                    "bytes_per_launch": dom_bytes, "us_per_launch": dom["us"]}
+                    "bytes_per_launch": dom_bytes, "us_per_launch": dom["us"],
+                    "target_frac": TARGET_GEMV_FRAC, "target_met": achieved / peaks["hbm_gbs"] >= TARGET_GEMV_FRAC}
 
         # end to end through the host-buffer entry point: pinned host x in, y out, every call
         xh = x.cpu().pin_memory()
@@ -389,7 +473,7 @@ def run_ours(args, rank, world):
         out = {"metric": "packed GEMV HBM GB/s (M=1 sweep, effective bytes K*N*(B+64/G)/8)", "value": round(value, 1),
                "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
                "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-               "dtype": "f16 tensor-core products of bf16 activations, fp32 accumulate",
+               "dtype": "f16 (bf16 activations rescaled to fp16 by a power of two; fp16 levels; fp16 group sums of 16 products, fp32 beyond)",
                "data": "synthetic: W ~ Laplace(0, 0.015) seed 1 encoded by cq_encode (fast effort), x ~ N(0,1) bf16",
                "config": {"workload": "gemv_sweep_8192", "M": 1, "N": N, "K": K, "B": SWEEP_B, "G": SWEEP_G,
                           "mode": "model_dtype", "l2": "each case rotates over copies totalling > 2x L2",
@@ -397,6 +481,13 @@ def run_ours(args, rank, world):
                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": n_launch,
                "clocks": clocks.summary(), "cases": per_case}
         out.update(extras)
+        # the summaries of the other kernels also ride inside the roofline object
+        for key in ("roofline_gemm", "roofline_a8", "config1_gemv_4096"):
+            if key in extras:
+                out["roofline"][key.replace("roofline_", "")] = extras[key]
+        if "decode_linears_w4g128" in extras:
+            out["roofline"]["decode_m1_frac_of_measured_hbm"] = {d["shape"]: d["frac_of_measured_hbm"]
+                                                                 for d in extras["decode_linears_w4g128"] if d["M"] == 1}
     if world > 1:
         dist.destroy_process_group()
     return out
@@ -461,8 +552,15 @@ def main():
                     help="sweep: headline GEMV sweep only; all: also prefill GEMM, decode linears, crossover")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        # not under torchrun: start the N replicas ourselves, one process per GPU
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", os.environ.get("MASTER_PORT", "29517"), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
+    if world != args.gpus:
+        sys.exit(f"--gpus {args.gpus} does not match WORLD_SIZE={world}")
     out = run_reference(args, rank, world) if args.impl == "reference" else run_ours(args, rank, world)
     if rank == 0 and out is not None:
         print(json.dumps(out), flush=True)
