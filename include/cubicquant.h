@@ -93,6 +93,13 @@ int cq_unpack(const void *layout, int B, int G, int64_t N, int64_t K, uint8_t *c
 int cq_gemm(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, int64_t M, int64_t N, int64_t K,
             int mode, void *workspace, size_t workspace_bytes, void *stream);
 
+/* The same product for a model whose dtype is IEEE binary16: x[M][K] and y[M][N] are binary16 bit patterns
+ * (Section 5.3: the model-dtype path accepts FP16 or BF16 activations).  Everything else -- arguments,
+ * modes, dispatch, workspace, errors -- is as for cq_gemm; in model-dtype mode the large-M kernel rounds its
+ * decoded weight tiles to binary16 instead of bfloat16, and both modes write y in binary16. */
+int cq_gemm_f16(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, int64_t M, int64_t N, int64_t K,
+                int mode, void *workspace, size_t workspace_bytes, void *stream);
+
 /* Reads back the device status word of a workspace (waits for `stream` first).  CQ_OK, or
  * CQ_ERR_TIMEOUT when a bounded device-side wait of an earlier cq_gemm on this workspace gave up
  * (its output is then undefined; re-initialise the workspace before reusing it). */
@@ -139,6 +146,8 @@ int cq_gemv_static(const void *layout, int B, int G, const uint16_t *x, uint16_t
  * x8[M][K] int8 and dx[M] float from x[M][K] bf16.  fp32 arithmetic: xbar = max(max|x|, 1e-10f),
  * dx = xbar / 127 (IEEE division), x8 = clip(round-half-away(x / dx), -127, 127). */
 int cq_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, float *dx, void *stream);
+/* The same quantiser for binary16 activations. */
+int cq_quantize_a8_f16(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, float *dx, void *stream);
 /* Non-negative reconstruction levels of every group (Appendix B): levels[N][K/G][L] float,
  * L = 2^(B-1) (W1: L = 1, the scale). */
 int cq_decode_levels(const void *layout, int B, int G, int64_t N, int64_t K, float *levels, void *stream);

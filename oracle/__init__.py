@@ -248,8 +248,9 @@ def _subset(idx):
     return arr, arr.size
 
 
-def gemm_model(codes, s, a, b, B, G, K, x_bf16, rows=None, cols=None) -> np.ndarray:
-    """fp64 y[rows, cols] of the model-dtype product; x_bf16 is uint16 bit patterns [M, K]."""
+def gemm_model(codes, s, a, b, B, G, K, x_bf16, rows=None, cols=None, act="bf16") -> np.ndarray:
+    """fp64 y[rows, cols] of the model-dtype product; x_bf16 is uint16 bit patterns [M, K] of the
+    activation dtype `act` ("bf16" or "f16")."""
     codes = _c(codes, np.uint8)
     s = _c(s, np.float32)
     a = _h(a)
@@ -261,17 +262,17 @@ def gemm_model(codes, s, a, b, B, G, K, x_bf16, rows=None, cols=None) -> np.ndar
     nr = nr if rows is not None else M
     nc = nc if cols is not None else N
     y = np.zeros((nr, nc), dtype=np.float64)
-    lib().cqo_gemm_model(_p(codes), _p(s), _p(a), _p(b), C.c_int(B), C.c_int(G), C.c_int64(N), C.c_int64(K), _p(x),
-                         C.c_int64(M), _p(r), C.c_int64(nr), _p(c), C.c_int64(nc), _p(y))
+    lib().cqo_gemm_model_act(_p(codes), _p(s), _p(a), _p(b), C.c_int(B), C.c_int(G), C.c_int64(N), C.c_int64(K), _p(x),
+                             C.c_int({"bf16": 0, "f16": 1}[act]), C.c_int64(M), _p(r), C.c_int64(nr), _p(c), C.c_int64(nc), _p(y))
     return y
 
 
-def quantize_a8(x_bf16):
+def quantize_a8(x_bf16, act="bf16"):
     x = _c(x_bf16, np.uint16)
     M, K = x.shape
     x8 = np.zeros((M, K), dtype=np.int8)
     dx = np.zeros(M, dtype=np.float32)
-    lib().cqo_quantize_a8(_p(x), C.c_int64(M), C.c_int64(K), _p(x8), _p(dx))
+    lib().cqo_quantize_a8_act(_p(x), C.c_int({"bf16": 0, "f16": 1}[act]), C.c_int64(M), C.c_int64(K), _p(x8), _p(dx))
     return x8, dx
 
 

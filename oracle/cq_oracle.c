@@ -75,6 +75,10 @@ static double bf16_to_double(uint16_t b) {
     return (double)f;
 }
 
+/* An activation's value from its 16-bit pattern: the model dtype is bfloat16 or binary16 (Section 5.3:
+ * the model-dtype path accepts FP16 or BF16 activations); both promote to double exactly. */
+static double act_to_double(uint16_t bits, int act_f16) { return act_f16 ? half_to_double(bits) : bf16_to_double(bits); }
+
 CQO_API double cqo_half_to_double(uint16_t h) { return half_to_double(h); }
 CQO_API uint16_t cqo_double_to_half(double d) { return double_to_half(d); }
 
@@ -609,9 +613,9 @@ CQO_API void cqo_encode_joint(const float *W, int64_t N, int64_t K, int B, int G
  * semantic reference of this mode.  x holds bfloat16 bit patterns (promoted exactly);
  * accumulation in fp64.  rows / cols select the activation rows m and output channels n to
  * evaluate (NULL = all); y is [nrows][ncols]. */
-CQO_API void cqo_gemm_model(const uint8_t *codes, const float *s, const uint16_t *a, const uint16_t *b, int B, int G,
-                            int64_t N, int64_t K, const uint16_t *x, int64_t M, const int64_t *rows, int64_t nrows,
-                            const int64_t *cols, int64_t ncols, double *y) {
+CQO_API void cqo_gemm_model_act(const uint8_t *codes, const float *s, const uint16_t *a, const uint16_t *b, int B, int G,
+                                int64_t N, int64_t K, const uint16_t *x, int act_f16, int64_t M, const int64_t *rows,
+                                int64_t nrows, const int64_t *cols, int64_t ncols, double *y) {
     int64_t ng = K / G;
     (void)N; (void)M;
 #pragma omp parallel
@@ -631,12 +635,18 @@ CQO_API void cqo_gemm_model(const uint8_t *codes, const float *s, const uint16_t
                 int64_t m = rows ? rows[ri] : ri;
                 const uint16_t *xr = x + m * K;
                 double acc = 0.0;
-                for (int64_t j = 0; j < K; ++j) acc += bf16_to_double(xr[j]) * wrow[j];
+                for (int64_t j = 0; j < K; ++j) acc += act_to_double(xr[j], act_f16) * wrow[j];
                 y[ri * ncols + ci] = acc;
             }
         }
         free(kk); free(wrow);
     }
+}
+
+CQO_API void cqo_gemm_model(const uint8_t *codes, const float *s, const uint16_t *a, const uint16_t *b, int B, int G,
+                            int64_t N, int64_t K, const uint16_t *x, int64_t M, const int64_t *rows, int64_t nrows,
+                            const int64_t *cols, int64_t ncols, double *y) {
+    cqo_gemm_model_act(codes, s, a, b, B, G, N, K, x, 0, M, rows, nrows, cols, ncols, y);   /* bfloat16 activations */
 }
 
 /* ------------------------------------------------------------------ Dynamic A8 (Section 5.4) */
@@ -645,25 +655,29 @@ CQO_API void cqo_gemm_model(const uint8_t *codes, const float *s, const uint16_t
  *   xbar = max(max_j |x_j|, eps),  d_x = xbar / 127,  x8_j = clip(round_away(x_j / d_x), -127, 127).
  * Bit-exact contract, so the arithmetic is pinned to fp32: eps = 1e-10f, both divisions are
  * IEEE fp32 divisions, roundf rounds halves away from zero. */
-CQO_API void cqo_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, float *dx) {
+CQO_API void cqo_quantize_a8_act(const uint16_t *x, int act_f16, int64_t M, int64_t K, int8_t *x8, float *dx) {
 #pragma omp parallel for schedule(static)
     for (int64_t m = 0; m < M; ++m) {
         float xbar = 0.0f;
         for (int64_t j = 0; j < K; ++j) {
-            float v = fabsf((float)bf16_to_double(x[m * K + j]));
+            float v = fabsf((float)act_to_double(x[m * K + j], act_f16));
             if (v > xbar) xbar = v;
         }
         if (!(xbar > 1e-10f)) xbar = 1e-10f;
         float d = xbar / 127.0f;
         dx[m] = d;
         for (int64_t j = 0; j < K; ++j) {
-            float v = (float)bf16_to_double(x[m * K + j]) / d;
+            float v = (float)act_to_double(x[m * K + j], act_f16) / d;
             float r = roundf(v);
             if (r > 127.0f) r = 127.0f;
             if (r < -127.0f) r = -127.0f;
             x8[m * K + j] = (int8_t)r;
         }
     }
+}
+
+CQO_API void cqo_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, float *dx) {
+    cqo_quantize_a8_act(x, 0, M, K, x8, dx);   /* bfloat16 activations */
 }
 
 /* Integer partials and output of the Dynamic-A8 product (Eq. a8-output):

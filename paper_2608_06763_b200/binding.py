@@ -49,6 +49,8 @@ def lib():
         L.cq_repack.argtypes = [vp, vp, vp, vp, i, i, i64, i64, vp, vp]
         L.cq_unpack.argtypes = [vp, i, i, i64, i64, vp, vp, vp, vp, vp]
         L.cq_gemm.argtypes = [vp, i, i, vp, vp, i64, i64, i64, i, vp, sz, vp]
+        L.cq_gemm_f16.argtypes = [vp, i, i, vp, vp, i64, i64, i64, i, vp, sz, vp]
+        L.cq_quantize_a8_f16.argtypes = [vp, i64, i64, vp, vp, vp]
         L.cq_gemm_status.argtypes = [vp, sz, vp]
         L.cq_gemm_status.restype = i
         L.cq_gemv_static.argtypes = [vp, i, i, vp, vp, i64, i64, i64, vp]
@@ -65,8 +67,8 @@ def lib():
         L.cq_encode_scale.argtypes = [vp, vp, i, i, i64, i64, vp, vp, i, vp, vp]
         L.cq_encode_losses.argtypes = [vp, vp, i, i, i64, i64, vp, vp, vp, vp, vp, vp]
         L.cq_encode.argtypes = [vp, i, i, i64, i64, i, i, vp, vp, vp, vp, vp]
-        for name in ("cq_workspace_init", "cq_pack_codes", "cq_repack", "cq_unpack", "cq_gemm", "cq_gemm_host",
-                     "cq_quantize_a8", "cq_decode_levels", "cq_decode_carriers", "cq_decode_weights",
+        for name in ("cq_workspace_init", "cq_pack_codes", "cq_repack", "cq_unpack", "cq_gemm", "cq_gemm_f16", "cq_gemm_host",
+                     "cq_quantize_a8", "cq_quantize_a8_f16", "cq_decode_levels", "cq_decode_carriers", "cq_decode_weights",
                      "cq_debug_a8_partials", "cq_encode_assign", "cq_encode_scale", "cq_encode_losses", "cq_encode"):
             getattr(L, name).restype = i
         _lib = L
@@ -156,13 +158,15 @@ def cq_unpack(pw: PackedWeights):
 
 def cq_gemm(pw: PackedWeights, x: torch.Tensor, mode: int = CQ_MODEL_DTYPE, workspace: torch.Tensor | None = None,
             out: torch.Tensor | None = None) -> torch.Tensor:
-    """y[M, N] bf16 = x[M, K] bf16 * What^T from the packed weights."""
-    assert x.dtype == torch.bfloat16 and x.dim() == 2 and x.shape[1] == pw.K
+    """y[M, N] = x[M, K] * What^T from the packed weights; x is bf16 or fp16 (the model dtype), y has the same dtype."""
+    assert x.dtype in (torch.bfloat16, torch.float16) and x.dim() == 2 and x.shape[1] == pw.K
     M = x.shape[0]
     if workspace is None:
         workspace = torch.zeros(cq_workspace_bytes(pw.B, pw.G, M, pw.N, pw.K, mode), dtype=torch.uint8, device=x.device)
-    y = out if out is not None else torch.empty((M, pw.N), dtype=torch.bfloat16, device=x.device)
-    _check(lib().cq_gemm(_ptr(pw.layout), pw.B, pw.G, _ptr(x), _ptr(y), M, pw.N, pw.K, mode, _ptr(workspace),
+    y = out if out is not None else torch.empty((M, pw.N), dtype=x.dtype, device=x.device)
+    assert y.dtype == x.dtype
+    fn = lib().cq_gemm if x.dtype == torch.bfloat16 else lib().cq_gemm_f16
+    _check(fn(_ptr(pw.layout), pw.B, pw.G, _ptr(x), _ptr(y), M, pw.N, pw.K, mode, _ptr(workspace),
                          workspace.numel(), _stream()), "cq_gemm")
     return y
 
@@ -198,7 +202,8 @@ def cq_quantize_a8(x: torch.Tensor):
     M, K = x.shape
     x8 = torch.empty((M, K), dtype=torch.int8, device=x.device)
     dx = torch.empty(M, dtype=torch.float32, device=x.device)
-    _check(lib().cq_quantize_a8(_ptr(x), M, K, _ptr(x8), _ptr(dx), _stream()), "cq_quantize_a8")
+    fn = lib().cq_quantize_a8 if x.dtype == torch.bfloat16 else lib().cq_quantize_a8_f16
+    _check(fn(_ptr(x), M, K, _ptr(x8), _ptr(dx), _stream()), "cq_quantize_a8")
     return x8, dx
 
 

@@ -137,8 +137,8 @@ int cq_unpack(const void *layout, int B, int G, int64_t N, int64_t K, uint8_t *c
     return wrap(launch_unpack(layout, make_dims(B, G, N, K), codes, scale, a, b, (cudaStream_t)stream));
 }
 
-int cq_gemm(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, int64_t M, int64_t N, int64_t K,
-            int mode, void *workspace, size_t workspace_bytes, void *stream) {
+static int gemm_any(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, int64_t M, int64_t N, int64_t K,
+                    int mode, bool act_f16, void *workspace, size_t workspace_bytes, void *stream) {
     if (!layout || !x || !y || !workspace || M <= 0) return CQ_ERR_INVALID_ARG;
     if (mode != CQ_MODEL_DTYPE && mode != CQ_DYN_A8) return CQ_ERR_INVALID_ARG;
     int st = check_format(B, G, N, K);
@@ -151,9 +151,19 @@ int cq_gemm(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, in
     if (st != CQ_OK) return st;
     cudaStream_t s = (cudaStream_t)stream;
     uint8_t *ws = (uint8_t *)workspace;
-    if (M <= 16) return wrap(launch_gemv(layout, d, x, y, M, mode, ws, plan, s));
-    if (mode == CQ_MODEL_DTYPE) return wrap(launch_gemm_tc(layout, d, x, y, M, mode, ws, plan, s));
-    return wrap(launch_gemm_a8_tc(layout, d, x, y, M, ws, plan, s));
+    if (M <= 16) return wrap(launch_gemv(layout, d, x, y, M, mode, act_f16, ws, plan, s));
+    if (mode == CQ_MODEL_DTYPE) return wrap(launch_gemm_tc(layout, d, x, y, M, mode, act_f16, ws, plan, s));
+    return wrap(launch_gemm_a8_tc(layout, d, x, y, M, act_f16, ws, plan, s));
+}
+
+int cq_gemm(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, int64_t M, int64_t N, int64_t K,
+            int mode, void *workspace, size_t workspace_bytes, void *stream) {
+    return gemm_any(layout, B, G, x, y, M, N, K, mode, false, workspace, workspace_bytes, stream);
+}
+
+int cq_gemm_f16(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, int64_t M, int64_t N, int64_t K,
+                int mode, void *workspace, size_t workspace_bytes, void *stream) {
+    return gemm_any(layout, B, G, x, y, M, N, K, mode, true, workspace, workspace_bytes, stream);
 }
 
 int cq_gemm_status(const void *workspace, size_t workspace_bytes, void *stream) {
@@ -222,7 +232,12 @@ int cq_encode(const float *W, int B, int G, int64_t N, int64_t K, int objective,
 
 int cq_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, float *dx, void *stream) {
     if (!x || !x8 || !dx || M <= 0 || K <= 0) return CQ_ERR_INVALID_ARG;
-    return wrap(launch_quantize_a8(x, M, K, x8, K, dx, false, (cudaStream_t)stream));
+    return wrap(launch_quantize_a8(x, M, K, x8, K, dx, false, false, (cudaStream_t)stream));
+}
+
+int cq_quantize_a8_f16(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, float *dx, void *stream) {
+    if (!x || !x8 || !dx || M <= 0 || K <= 0) return CQ_ERR_INVALID_ARG;
+    return wrap(launch_quantize_a8(x, M, K, x8, K, dx, false, true, (cudaStream_t)stream));
 }
 
 #define CQ_DEBUG_PROLOGUE()                                   \

@@ -119,6 +119,29 @@ __host__ __device__ inline void weight_of(int rb, int lane, int pair, int half, 
     kk = 16 * j + 4 * t + (i >> 1) * 2 + half;
 }
 
+// ---- activations / outputs in the model dtype: bfloat16 or binary16 bit patterns (Section 5.3) ----------
+// value of one 16-bit activation pattern
+__device__ __forceinline__ float act_to_float(uint32_t bits16, bool f16) {
+    return f16 ? __half2float(__ushort_as_half((unsigned short)bits16)) : __uint_as_float(bits16 << 16);
+}
+// fp32 -> the output dtype, round to nearest even
+__device__ __forceinline__ uint16_t float_to_act(float v, bool f16) {
+    return f16 ? __half_as_ushort(__float2half_rn(v)) : __bfloat16_as_ushort(__float2bfloat16_rn(v));
+}
+// Power-of-two exponent e with |x| < 2^(e+1) for the largest magnitude pattern of a row (sign cleared; for
+// finite values the integer order of the patterns is the order of the magnitudes).  `usable` is false for
+// an all-zero row and for Inf / NaN (no rescaling then).
+__device__ __forceinline__ int act_max_exponent(unsigned max_bits, bool f16, bool &usable) {
+    if (f16) {
+        const int ef = (int)((max_bits >> 10) & 0x1F);
+        usable = max_bits != 0 && ef != 31;
+        return (ef == 0 ? 1 : ef) - 15;          // subnormals count as 2^-14
+    }
+    const int ef = (int)((max_bits >> 7) & 0xFF);
+    usable = max_bits != 0 && ef != 255;
+    return ef - 127;
+}
+
 struct __align__(8) GroupParams { float s; __half a; __half b; };
 
 __device__ __forceinline__ const uint8_t *tile_ptr(const void *layout, const Dims &d, int nb, int kb) {

@@ -59,6 +59,7 @@ struct A8Params {
     int raw_stage_bytes;
     float *partial;       // split-K: fp32 partial sums [SK][M][Np] (before the d_x / 127 factor)
     int *counters;        // split-K: arrival counters, one per (row block, token tile)
+    bool f16;             // y is written as binary16 instead of bfloat16
 };
 
 __device__ __forceinline__ void named_barrier_sync(int id, int threads) {
@@ -303,7 +304,7 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
                     if (m < prm.M) {
                         if (gridDim.z == 1) {
                             const float v = acc[i] * (prm.dx[m] * (1.0f / 127.0f));
-                            prm.y[m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+                            prm.y[m * d.N + n] = float_to_act(v, prm.f16);
                         } else {
                             prm.partial[((size_t)blockIdx.z * prm.M + m) * ((size_t)d.NB * TILE) + n] = acc[i];
                         }
@@ -348,7 +349,7 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
                 const float o[4] = {sum.x * f, sum.y * f, sum.z * f, sum.w * f};
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                    if (n + e < d.N) prm.y[m * d.N + n + e] = __bfloat16_as_ushort(__float2bfloat16_rn(o[e]));
+                    if (n + e < d.N) prm.y[m * d.N + n + e] = float_to_act(o[e], prm.f16);
             }
             if (threadIdx.x == 0) *ctr = 0;  // leave the workspace ready for the next call
         }
@@ -357,7 +358,7 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
 
 template <int B, int G, int BN>
 cudaError_t launch_a8(const void *layout, const Dims &d, const int8_t *x8, int64_t pitch, const float *dx, uint16_t *y,
-                      int64_t M, int *status, float *partial, int *counters, cudaStream_t st) {
+                      int64_t M, int *status, float *partial, int *counters, bool act_f16, cudaStream_t st) {
     constexpr int GPT = TILE / G;
     EncodeTiledFn enc = encode_tiled();
     if (!enc) return cudaErrorNotSupported;
@@ -372,7 +373,7 @@ cudaError_t launch_a8(const void *layout, const Dims &d, const int8_t *x8, int64
         return cudaErrorInvalidValue;
     A8Params p;
     p.layout = (const uint8_t *)layout; p.dx = dx; p.y = y; p.status = status; p.d = d; p.M = (int)M;
-    p.partial = partial; p.counters = counters;
+    p.partial = partial; p.counters = counters; p.f16 = act_f16;
     p.raw_stage_bytes = (d.tile_bytes + 1023) / 1024 * 1024;
     const size_t smem = (size_t)A8_STAGES * (A8_A_STAGE_BYTES + BN * 128) + (size_t)A8_RAW_STAGES * p.raw_stage_bytes +
                         (size_t)8 * 2 * 16 * carrier_table_stride(B) + (size_t)A8_SRING * 128 * GPT * 4 + 512 + 256;
@@ -388,46 +389,46 @@ cudaError_t launch_a8(const void *layout, const Dims &d, const int8_t *x8, int64
 // token tile: two accumulator buffers of GPT x BN columns must fit the 512 TMEM columns
 template <int B, int G>
 cudaError_t launch_a8_bn(const void *layout, const Dims &d, const int8_t *x8, int64_t pitch, const float *dx, uint16_t *y,
-                         int64_t M, int *status, float *partial, int *counters, cudaStream_t st) {
+                         int64_t M, int *status, float *partial, int *counters, bool act_f16, cudaStream_t st) {
     constexpr int BMAX = 256 / (TILE / G);
     const int bn = gemm_a8_token_tile(d, M);
-    if constexpr (BMAX >= 256) if (bn == 256) return launch_a8<B, G, 256>(layout, d, x8, pitch, dx, y, M, status, partial, counters, st);
-    if constexpr (BMAX >= 128) if (bn == 128) return launch_a8<B, G, 128>(layout, d, x8, pitch, dx, y, M, status, partial, counters, st);
-    return launch_a8<B, G, 64>(layout, d, x8, pitch, dx, y, M, status, partial, counters, st);
+    if constexpr (BMAX >= 256) if (bn == 256) return launch_a8<B, G, 256>(layout, d, x8, pitch, dx, y, M, status, partial, counters, act_f16, st);
+    if constexpr (BMAX >= 128) if (bn == 128) return launch_a8<B, G, 128>(layout, d, x8, pitch, dx, y, M, status, partial, counters, act_f16, st);
+    return launch_a8<B, G, 64>(layout, d, x8, pitch, dx, y, M, status, partial, counters, act_f16, st);
 }
 
 template <int B>
 cudaError_t launch_a8_b(const void *layout, const Dims &d, const int8_t *x8, int64_t pitch, const float *dx, uint16_t *y,
-                        int64_t M, int *status, float *partial, int *counters, cudaStream_t st) {
+                        int64_t M, int *status, float *partial, int *counters, bool act_f16, cudaStream_t st) {
     switch (d.G) {
-        case 32: return launch_a8_bn<B, 32>(layout, d, x8, pitch, dx, y, M, status, partial, counters, st);
-        case 64: return launch_a8_bn<B, 64>(layout, d, x8, pitch, dx, y, M, status, partial, counters, st);
-        default: return launch_a8_bn<B, 128>(layout, d, x8, pitch, dx, y, M, status, partial, counters, st);
+        case 32: return launch_a8_bn<B, 32>(layout, d, x8, pitch, dx, y, M, status, partial, counters, act_f16, st);
+        case 64: return launch_a8_bn<B, 64>(layout, d, x8, pitch, dx, y, M, status, partial, counters, act_f16, st);
+        default: return launch_a8_bn<B, 128>(layout, d, x8, pitch, dx, y, M, status, partial, counters, act_f16, st);
     }
 }
 
 }  // namespace
 
 // Quantise the activations (one block per row), then run the tcgen05 INT8 GEMM on the carriers.
-cudaError_t launch_gemm_a8_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, uint8_t *ws,
-                              const Workspace &plan, cudaStream_t st) {
+cudaError_t launch_gemm_a8_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, bool act_f16,
+                              uint8_t *ws, const Workspace &plan, cudaStream_t st) {
     int8_t *xq = reinterpret_cast<int8_t *>(ws + plan.x8_off);
     float *dxs = reinterpret_cast<float *>(ws + plan.dx_off);
     int *status = reinterpret_cast<int *>(ws + plan.status_off);
     float *partial = reinterpret_cast<float *>(ws + plan.partial_off);
     int *counters = reinterpret_cast<int *>(ws + plan.counters_off);
     const int64_t pitch = (int64_t)d.KT * TILE;
-    cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, true, st);
+    cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, true, act_f16, st);
     if (e != cudaSuccess) return e;
     switch (d.B) {
-        case 1: return launch_a8_b<1>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
-        case 2: return launch_a8_b<2>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
-        case 3: return launch_a8_b<3>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
-        case 4: return launch_a8_b<4>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
-        case 5: return launch_a8_b<5>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
-        case 6: return launch_a8_b<6>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
-        case 7: return launch_a8_b<7>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
-        default: return launch_a8_b<8>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, st);
+        case 1: return launch_a8_b<1>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, act_f16, st);
+        case 2: return launch_a8_b<2>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, act_f16, st);
+        case 3: return launch_a8_b<3>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, act_f16, st);
+        case 4: return launch_a8_b<4>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, act_f16, st);
+        case 5: return launch_a8_b<5>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, act_f16, st);
+        case 6: return launch_a8_b<6>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, act_f16, st);
+        case 7: return launch_a8_b<7>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, act_f16, st);
+        default: return launch_a8_b<8>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, act_f16, st);
     }
 }
 

@@ -50,27 +50,35 @@ constexpr int RAW_STAGES = 2;
 // Two reconstructed weights s * sign(k) * q(|k| / M) of one pair, rounded to bf16 (the dense path
 // of Section 5.3 rounds the temporary operand to the activation dtype).  q is evaluated in half2
 // (11-bit significand, finer than the bf16 it is rounded to), the scale is applied in fp32.
-template <int B, int P, bool FIX>
+template <int B, int P, bool FIX, bool F16>
 __device__ __forceinline__ uint32_t weight_pair_bf16(const uint32_t (&w)[2 * B], const RowCoef &c) {
     const __half2 T = pair_T<B, P>(w);
     const uint32_t q = level_pair<B, FIX>(T, c);
     const float2 f = __half22float2(as_h2(q));
-    const __nv_bfloat162 v = __floats2bfloat162_rn(f.x * c.s, f.y * c.s);
-    return *reinterpret_cast<const uint32_t *>(&v);
+    if constexpr (F16) {   // binary16 activations: the temporary operand is rounded to binary16
+        return as_u32(__floats2half2_rn(f.x * c.s, f.y * c.s));
+    } else {
+        const __nv_bfloat162 v = __floats2bfloat162_rn(f.x * c.s, f.y * c.s);
+        return *reinterpret_cast<const uint32_t *>(&v);
+    }
 }
 
 // W3: the eight stored codes of a (row, group) index a signed bf16 table of s * sign(k) * q(|k| / 3)
 // (u = 0, the reserved pattern, and k = 0 read zero), kept as a low-byte and a high-byte register pair
 // and read four codes at a time with byte permutes; q(1/3) and q(2/3) by the fp32 Horner form.
 struct W3Table { uint32_t lo[2], hi[2]; };
-__device__ __forceinline__ W3Table w3_table(uint2 p) {
+__device__ __forceinline__ uint32_t pack_act2(float lo, float hi, bool f16) {   // two values in the activation dtype
+    if (f16) return as_u32(__floats2half2_rn(lo, hi));
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&v);
+}
+__device__ __forceinline__ W3Table w3_table(uint2 p, bool f16) {
     const float s = __uint_as_float(p.x & 0x7FFFFFFFu);
     const __half2 ab = as_h2(p.y);
     const float a = __low2float(ab), b = __high2float(ab), c = (1.0f - a) - b;
     constexpr float t1 = 1.0f / 3.0f, t2 = 2.0f / 3.0f;
     const float q1 = t1 * fmaf(t1, fmaf(t1, c, b), a), q2 = t2 * fmaf(t2, fmaf(t2, c, b), a);
-    const __nv_bfloat162 v12 = __floats2bfloat162_rn(s * q1, s * q2), vs = __floats2bfloat162_rn(s, 0.0f);
-    const uint32_t q12 = *reinterpret_cast<const uint32_t *>(&v12), ss = *reinterpret_cast<const uint32_t *>(&vs);
+    const uint32_t q12 = pack_act2(s * q1, s * q2, f16), ss = pack_act2(s, 0.0f, f16);
     const uint32_t nq = q12 | 0x80008000u, ns = ss | 0x00008000u;
     W3Table t;                                  // entries u = 0 .. 7:  0, -s, -s q2, -s q1 | 0, s q1, s q2, s
     t.lo[0] = prmt(nq, ns, 0x0247u) & 0xFFFFFF00u;   // low bytes:  0, (-s).lo, (-s q2).lo, (-s q1).lo
@@ -106,6 +114,7 @@ struct TcParams {
     int raw_stage_bytes;  // tile_bytes rounded up to 1024
     float *partial;       // split-K: fp32 partial sums [SK][M][Np]
     int *counters;        // split-K: arrival counters, one per (row block, token tile)
+    bool f16;             // activations and output are binary16 instead of bfloat16 (the weights are decoded to match)
 };
 
 // ---------------------------------------------------------------- the kernel (model dtype)
@@ -183,7 +192,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
     } else if (warp == 1) {
         // ===== MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16(BN);
+            const uint32_t idesc = prm.f16 ? idesc_f16(BN) : idesc_bf16(BN);
             bool ok = true;
             for (int kb = 0; kb < NKB && ok; ++kb) {
                 const int s = kb % STAGES;
@@ -231,8 +240,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
             const uint8_t *prow = raw + d.code_bytes + ((rb * 16 + g) * GPT) * 8;
             W3Table w3_lo{}, w3_hi{};   // W3: level tables of rows g and g + 8; one per tile when the group spans it
             if constexpr (B == 3 && G == 128) {
-                w3_lo = w3_table(*(const uint2 *)prow);
-                w3_hi = w3_table(*(const uint2 *)(prow + 8 * GPT * 8));
+                w3_lo = w3_table(*(const uint2 *)prow, prm.f16);
+                w3_hi = w3_table(*(const uint2 *)(prow + 8 * GPT * 8), prm.f16);
             }
 #pragma unroll 1
             for (int half_k = 0; half_k < 2 && ok; ++half_k) {
@@ -249,7 +258,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                     const uint2 p_lo = *(const uint2 *)(prow + gi * 8), p_hi = *(const uint2 *)(prow + (8 * GPT + gi) * 8);
                     if constexpr (B == 3) {
                         // table decode (w3_block): no per-weight arithmetic, the reserved pattern reads zero
-                        if constexpr (G < 128) { w3_lo = w3_table(p_lo); w3_hi = w3_table(p_hi); }
+                        if constexpr (G < 128) { w3_lo = w3_table(p_lo, prm.f16); w3_hi = w3_table(p_hi, prm.f16); }
                         uint32_t o_lo[4], o_hi[4];
                         w3_block<0, JQ>(w, w3_lo, o_lo);
                         w3_block<1, JQ>(w, w3_hi, o_hi);
@@ -263,15 +272,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                     }
                     const RowCoef c_lo = make_coef<B>(p_lo), c_hi = make_coef<B>(p_hi);
                     const bool fix = B > 1 && __any_sync(0xffffffffu, (p_lo.x | p_hi.x) >> 31);  // reserved pattern present
-                    auto emit = [&](auto fx) {
-                        constexpr bool FIX = decltype(fx)::value;
+                    auto emit = [&](auto fx, auto hx) {
+                        constexpr bool FIX = decltype(fx)::value, F16 = decltype(hx)::value;
                         static_for<2>([&](auto jc) {
                             constexpr int j = 2 * JQ + decltype(jc)::value, jl = j & 3;
                             uint2 lo, hi;  // four consecutive k of one row = 8 bytes
-                            lo.x = weight_pair_bf16<B, 4 * j + 0, FIX>(w, c_lo);
-                            hi.x = weight_pair_bf16<B, 4 * j + 1, FIX>(w, c_hi);
-                            lo.y = weight_pair_bf16<B, 4 * j + 2, FIX>(w, c_lo);
-                            hi.y = weight_pair_bf16<B, 4 * j + 3, FIX>(w, c_hi);
+                            lo.x = weight_pair_bf16<B, 4 * j + 0, FIX, F16>(w, c_lo);
+                            hi.x = weight_pair_bf16<B, 4 * j + 1, FIX, F16>(w, c_hi);
+                            lo.y = weight_pair_bf16<B, 4 * j + 2, FIX, F16>(w, c_lo);
+                            hi.y = weight_pair_bf16<B, 4 * j + 3, FIX, F16>(w, c_hi);
                             // k offset inside the 64-wide block: 16 jl + 4 t -> 16-byte chunk 2 jl + t/2, swizzled by the row
                             const int chunk = (2 * jl + (t >> 1)) ^ g;
                             const int off = chunk * 16 + (t & 1) * 8;
@@ -279,7 +288,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                             *(uint2 *)(row_hi + off) = hi;
                         });
                     };
-                    if (!fix) emit(std::false_type{}); else emit(std::true_type{});
+                    if (!prm.f16) { if (!fix) emit(std::false_type{}, std::false_type{}); else emit(std::true_type{}, std::false_type{}); }
+                    else { if (!fix) emit(std::false_type{}, std::true_type{}); else emit(std::true_type{}, std::true_type{}); }
                 };
                 switch (half_k * 2 + jh) {
                     case 0: do_unit(std::integral_constant<int, 0>{}); break;
@@ -311,7 +321,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                     for (int i = 0; i < 32; ++i) {
                         const int64_t m = (int64_t)mt * BNT + c0 + i;
                         if (m < prm.M) {
-                            if (gridDim.z == 1) prm.y[m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(r[i])));
+                            if (gridDim.z == 1) prm.y[m * d.N + n] = float_to_act(__uint_as_float(r[i]), prm.f16);
                             else prm.partial[((size_t)blockIdx.z * prm.M + m) * ((size_t)d.NB * TILE) + n] = __uint_as_float(r[i]);
                         }
                     }
@@ -367,7 +377,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                     const float o[4] = {sum.x, sum.y, sum.z, sum.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
-                        if (n + e < d.N) prm.y[m * d.N + n + e] = __bfloat16_as_ushort(__float2bfloat16_rn(o[e]));
+                        if (n + e < d.N) prm.y[m * d.N + n + e] = float_to_act(o[e], prm.f16);
                 }
             }
             if (threadIdx.x == 0) *ctr = 0;  // leave the workspace ready for the next call
@@ -378,7 +388,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
 // ---------------------------------------------------------------- host side
 template <int B, int G, int BN, int NACC>
 cudaError_t launch_bn(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int *status,
-                      float *partial, int *counters, cudaStream_t st) {
+                      float *partial, int *counters, bool act_f16, cudaStream_t st) {
     EncodeTiledFn enc = encode_tiled();
     if (!enc) return cudaErrorNotSupported;
     CUtensorMap xmap;
@@ -386,7 +396,7 @@ cudaError_t launch_bn(const void *layout, const Dims &d, const uint16_t *x, uint
     const cuuint64_t strides[1] = {(cuuint64_t)d.K * 2};
     const cuuint32_t box[2] = {64, (cuuint32_t)BN};
     const cuuint32_t estr[2] = {1, 1};
-    if (enc(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t *>(x), dims, strides, box, estr,
+    if (enc(&xmap, act_f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t *>(x), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
@@ -399,7 +409,7 @@ cudaError_t launch_bn(const void *layout, const Dims &d, const uint16_t *x, uint
     static std::atomic<uint64_t> attr_done{0};   // per kernel instantiation: the devices it has been set on
     cudaError_t ea = ensure_func_attr(kern, attr_done, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (ea != cudaSuccess) return ea;
-    p.partial = partial; p.counters = counters;
+    p.partial = partial; p.counters = counters; p.f16 = act_f16;
     dim3 grid((unsigned)d.NB, (unsigned)((M + BN * NACC - 1) / (BN * NACC)), (unsigned)gemm_tc_split_k(d, M));
     kern<<<grid, TC_THREADS, smem, st>>>(xmap, p);
     return cudaGetLastError();
@@ -407,41 +417,41 @@ cudaError_t launch_bn(const void *layout, const Dims &d, const uint16_t *x, uint
 
 template <int B, int G>
 cudaError_t launch_g(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int *status,
-                     float *partial, int *counters, cudaStream_t st) {
-    if (M <= 32) return launch_bn<B, G, 32, 1>(layout, d, x, y, M, status, partial, counters, st);
-    if (M <= 64) return launch_bn<B, G, 64, 1>(layout, d, x, y, M, status, partial, counters, st);
-    if (M <= 128) return launch_bn<B, G, 128, 1>(layout, d, x, y, M, status, partial, counters, st);
-    if (M <= 256) return launch_bn<B, G, 256, 1>(layout, d, x, y, M, status, partial, counters, st);
-    return launch_bn<B, G, 256, 2>(layout, d, x, y, M, status, partial, counters, st);
+                     float *partial, int *counters, bool act_f16, cudaStream_t st) {
+    if (M <= 32) return launch_bn<B, G, 32, 1>(layout, d, x, y, M, status, partial, counters, act_f16, st);
+    if (M <= 64) return launch_bn<B, G, 64, 1>(layout, d, x, y, M, status, partial, counters, act_f16, st);
+    if (M <= 128) return launch_bn<B, G, 128, 1>(layout, d, x, y, M, status, partial, counters, act_f16, st);
+    if (M <= 256) return launch_bn<B, G, 256, 1>(layout, d, x, y, M, status, partial, counters, act_f16, st);
+    return launch_bn<B, G, 256, 2>(layout, d, x, y, M, status, partial, counters, act_f16, st);
 }
 
 template <int B>
 cudaError_t launch_b(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int *status,
-                     float *partial, int *counters, cudaStream_t st) {
+                     float *partial, int *counters, bool act_f16, cudaStream_t st) {
     switch (d.G) {
-        case 32: return launch_g<B, 32>(layout, d, x, y, M, status, partial, counters, st);
-        case 64: return launch_g<B, 64>(layout, d, x, y, M, status, partial, counters, st);
-        default: return launch_g<B, 128>(layout, d, x, y, M, status, partial, counters, st);
+        case 32: return launch_g<B, 32>(layout, d, x, y, M, status, partial, counters, act_f16, st);
+        case 64: return launch_g<B, 64>(layout, d, x, y, M, status, partial, counters, act_f16, st);
+        default: return launch_g<B, 128>(layout, d, x, y, M, status, partial, counters, act_f16, st);
     }
 }
 
 }  // namespace
 
 cudaError_t launch_gemm_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
-                           uint8_t *ws, const Workspace &plan, cudaStream_t st) {
+                           bool act_f16, uint8_t *ws, const Workspace &plan, cudaStream_t st) {
     if (mode != 0) return cudaErrorNotSupported;
     int *status = reinterpret_cast<int *>(ws + plan.status_off);
     float *partial = reinterpret_cast<float *>(ws + plan.partial_off);
     int *counters = reinterpret_cast<int *>(ws + plan.counters_off);
     switch (d.B) {
-        case 1: return launch_b<1>(layout, d, x, y, M, status, partial, counters, st);
-        case 2: return launch_b<2>(layout, d, x, y, M, status, partial, counters, st);
-        case 3: return launch_b<3>(layout, d, x, y, M, status, partial, counters, st);
-        case 4: return launch_b<4>(layout, d, x, y, M, status, partial, counters, st);
-        case 5: return launch_b<5>(layout, d, x, y, M, status, partial, counters, st);
-        case 6: return launch_b<6>(layout, d, x, y, M, status, partial, counters, st);
-        case 7: return launch_b<7>(layout, d, x, y, M, status, partial, counters, st);
-        default: return launch_b<8>(layout, d, x, y, M, status, partial, counters, st);
+        case 1: return launch_b<1>(layout, d, x, y, M, status, partial, counters, act_f16, st);
+        case 2: return launch_b<2>(layout, d, x, y, M, status, partial, counters, act_f16, st);
+        case 3: return launch_b<3>(layout, d, x, y, M, status, partial, counters, act_f16, st);
+        case 4: return launch_b<4>(layout, d, x, y, M, status, partial, counters, act_f16, st);
+        case 5: return launch_b<5>(layout, d, x, y, M, status, partial, counters, act_f16, st);
+        case 6: return launch_b<6>(layout, d, x, y, M, status, partial, counters, act_f16, st);
+        case 7: return launch_b<7>(layout, d, x, y, M, status, partial, counters, act_f16, st);
+        default: return launch_b<8>(layout, d, x, y, M, status, partial, counters, act_f16, st);
     }
 }
 

@@ -495,7 +495,7 @@ template <int B, int G, int NT, int MODE>
 __global__ void __launch_bounds__(GEMV_THREADS, gemv_occ(B, G, NT, MODE))
 gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restrict__ x, const int8_t *__restrict__ xq,
             int64_t x8_pitch, const float *__restrict__ dxs, uint16_t *__restrict__ y, int M, int E,
-            float *__restrict__ partial, int *__restrict__ counters, int nstage, uint32_t ring_off, int *__restrict__ status) {
+            float *__restrict__ partial, int *__restrict__ counters, int nstage, uint32_t ring_off, int *__restrict__ status, bool xf16) {
     constexpr int GPT = TILE / G;
     constexpr int L = B == 1 ? 1 : (1 << (B - 1));
     constexpr bool RING = gemv_uses_ring(B, G, NT, MODE);
@@ -652,8 +652,9 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                 // [2^14, 2^15) (MODE 2: [2^10, 2^11), its sums stay in fp16) and converts the chunks it owns
                 auto convert_row = [&](int m) {
                     const unsigned mb = s_max[m];
-                    const int ef = (int)((mb >> 7) & 0xFF);          // biased exponent of the maximum
-                    int sh = (mb == 0 || ef == 255) ? 0 : (MODE == 2 ? 10 : 14) - ef + 127;
+                    bool usable;
+                    const int e_max = act_max_exponent(mb, xf16, usable);   // the row maximum lies in [2^e_max, 2^(e_max+1))
+                    int sh = usable ? (MODE == 2 ? 10 : 14) - e_max : 0;
                     sh = max(min(sh, 100), -100);
                     const float sc = __uint_as_float((uint32_t)(127 + sh) << 23);   // 2^sh
                     if (threadIdx.x == m) s_inv[m] = __uint_as_float((uint32_t)(127 - sh) << 23);
@@ -663,7 +664,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                         ws[0] = v4.x; ws[1] = v4.y; ws[2] = v4.z; ws[3] = v4.w;
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
-                            const float lo = __uint_as_float(ws[q] << 16) * sc, hi = __uint_as_float(ws[q] & 0xFFFF0000u) * sc;
+                            const float lo = act_to_float(ws[q] & 0xFFFFu, xf16) * sc, hi = act_to_float(ws[q] >> 16, xf16) * sc;
                             ws[q] = as_u32(__floats2half2_rn(lo, hi));
                         }
                     }
@@ -792,7 +793,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                 if (tok >= M) continue;
                 if (whole) {
                     const int64_t n = n_lo + ((i >> 1) ? 8 : 0);
-                    if (n < d.N) y[(int64_t)tok * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(total[tb][i]));
+                    if (n < d.N) y[(int64_t)tok * d.N + n] = float_to_act(total[tb][i], xf16);
                 } else {
                     pslot[tok * TILE + r] = total[tb][i];
                 }
@@ -827,7 +828,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
 #pragma unroll
                             for (int i = 0; i < 8; ++i) sum += vv[i];
                         }
-                        if (n < d.N) y[(int64_t)m * d.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(sum));
+                        if (n < d.N) y[(int64_t)m * d.N + n] = float_to_act(sum, xf16);
                     }
                 } else {
                     // four consecutive channels of one token per thread and step (128-bit loads), up to eight
@@ -850,7 +851,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
                         const float o[4] = {sum.x, sum.y, sum.z, sum.w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e)
-                            if (n + e < d.N) y[(int64_t)m * d.N + n + e] = __bfloat16_as_ushort(__float2bfloat16_rn(o[e]));
+                            if (n + e < d.N) y[(int64_t)m * d.N + n + e] = float_to_act(o[e], xf16);
                     }
                 }
                 if (threadIdx.x == 0) counters[nb] = 0;  // leave the workspace ready for the next call
@@ -867,7 +868,7 @@ gemv_kernel(const uint8_t *__restrict__ layout, Dims d, const uint16_t *__restri
 template <int B, int G, int NT, int MODE>
 cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, const int8_t *xq, int64_t x8_pitch,
                        const float *dxs, uint16_t *y, int M, int P, int max_run, int E, float *partial, int *counters,
-                       int *status, cudaStream_t st) {
+                       int *status, bool act_f16, cudaStream_t st) {
     constexpr int GPT = TILE / G;
     constexpr int TB = 2048 * B + 1024 * GPT;
     int64_t sub64 = max_run;   // the longest run bounds the activation slice a CTA stages
@@ -904,31 +905,31 @@ cudaError_t launch_one(const void *layout, const Dims &d, const uint16_t *x, con
     cfg.attrs = attr;
     cfg.numAttrs = use_pdl ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kern, (const uint8_t *)layout, d, x, xq, x8_pitch, dxs, y, M, E, partial, counters, nstage,
-                              ring_off, status);
+                              ring_off, status, act_f16);
 }
 
 template <int B, int G>
 cudaError_t dispatch_nt_mode(const void *layout, const Dims &d, const uint16_t *x, const int8_t *xq, int64_t x8_pitch,
                              const float *dxs, uint16_t *y, int M, int mode, int P, int max_run, int E, float *partial,
-                             int *counters, int *status, cudaStream_t st) {
+                             int *counters, int *status, bool act_f16, cudaStream_t st) {
     if (mode == 0) {
-        if (M == 1) return launch_one<B, G, 1, 2>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, status, st);
-        if (M == 2) return launch_one<B, G, 2, 2>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, status, st);
-        if (M <= 8) return launch_one<B, G, 1, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, status, st);
-        return launch_one<B, G, 2, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, status, st);
+        if (M == 1) return launch_one<B, G, 1, 2>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, status, act_f16, st);
+        if (M == 2) return launch_one<B, G, 2, 2>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, status, act_f16, st);
+        if (M <= 8) return launch_one<B, G, 1, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, status, act_f16, st);
+        return launch_one<B, G, 2, 0>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, status, act_f16, st);
     }
-    if (M <= 8) return launch_one<B, G, 1, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, status, st);
-    return launch_one<B, G, 2, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, status, st);
+    if (M <= 8) return launch_one<B, G, 1, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, status, act_f16, st);
+    return launch_one<B, G, 2, 1>(layout, d, x, xq, x8_pitch, dxs, y, M, P, max_run, E, partial, counters, status, act_f16, st);
 }
 
 template <int B>
 cudaError_t dispatch_g(const void *layout, const Dims &d, const uint16_t *x, const int8_t *xq, int64_t x8_pitch,
                        const float *dxs, uint16_t *y, int M, int mode, int P, int max_run, int E, float *partial,
-                       int *counters, int *status, cudaStream_t st) {
+                       int *counters, int *status, bool act_f16, cudaStream_t st) {
     switch (d.G) {
-        case 32: return dispatch_nt_mode<B, 32>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_run, E, partial, counters, status, st);
-        case 64: return dispatch_nt_mode<B, 64>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_run, E, partial, counters, status, st);
-        default: return dispatch_nt_mode<B, 128>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_run, E, partial, counters, status, st);
+        case 32: return dispatch_nt_mode<B, 32>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_run, E, partial, counters, status, act_f16, st);
+        case 64: return dispatch_nt_mode<B, 64>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_run, E, partial, counters, status, act_f16, st);
+        default: return dispatch_nt_mode<B, 128>(layout, d, x, xq, x8_pitch, dxs, y, M, mode, P, max_run, E, partial, counters, status, act_f16, st);
     }
 }
 
@@ -962,7 +963,7 @@ GemvPlan gemv_plan(const Dims &d, int64_t M, int mode) {
 }
 
 cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
-                        uint8_t *ws, const Workspace &plan, cudaStream_t st) {
+                        bool act_f16, uint8_t *ws, const Workspace &plan, cudaStream_t st) {
     const GemvPlan gp = gemv_plan(d, M, mode);
     float *partial = reinterpret_cast<float *>(ws + plan.partial_off);
     int *counters = reinterpret_cast<int *>(ws + plan.counters_off);
@@ -971,27 +972,27 @@ cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, ui
     float *dxs = reinterpret_cast<float *>(ws + plan.dx_off);
     const int64_t pitch = (int64_t)d.KT * TILE;
     if (mode == 1) {
-        cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, true, st);
+        cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, true, act_f16, st);
         if (e != cudaSuccess) return e;
     }
     const int Mi = (int)M, P = gp.ctas, ms = gp.max_run;
     const int E = gp.overhead;
 #ifdef CQ_GEMV_SUBSET   // development builds: only the widths under study
     switch (d.B) {
-        case 1: return dispatch_g<1>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, st);
-        case 4: return dispatch_g<4>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, st);
+        case 1: return dispatch_g<1>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, act_f16, st);
+        case 4: return dispatch_g<4>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, act_f16, st);
         default: return cudaErrorNotSupported;
     }
 #else
     switch (d.B) {
-        case 1: return dispatch_g<1>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, st);
-        case 2: return dispatch_g<2>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, st);
-        case 3: return dispatch_g<3>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, st);
-        case 4: return dispatch_g<4>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, st);
-        case 5: return dispatch_g<5>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, st);
-        case 6: return dispatch_g<6>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, st);
-        case 7: return dispatch_g<7>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, st);
-        default: return dispatch_g<8>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, st);
+        case 1: return dispatch_g<1>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, act_f16, st);
+        case 2: return dispatch_g<2>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, act_f16, st);
+        case 3: return dispatch_g<3>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, act_f16, st);
+        case 4: return dispatch_g<4>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, act_f16, st);
+        case 5: return dispatch_g<5>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, act_f16, st);
+        case 6: return dispatch_g<6>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, act_f16, st);
+        case 7: return dispatch_g<7>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, act_f16, st);
+        default: return dispatch_g<8>(layout, d, x, xq, pitch, dxs, y, Mi, mode, P, ms, E, partial, counters, status, act_f16, st);
     }
 #endif
 }

@@ -18,8 +18,9 @@ cudaError_t launch_decode_levels(const void *layout, const Dims &d, float *level
 cudaError_t launch_decode_carriers(const void *layout, const Dims &d, int8_t *carriers, cudaStream_t st);
 cudaError_t launch_decode_weights(const void *layout, const Dims &d, float *What, cudaStream_t st);
 cudaError_t launch_a8_partials(const void *layout, const Dims &d, const int8_t *x8, int64_t M, int32_t *P, cudaStream_t st);
+// act_f16 (here and below): the 16-bit activation / output patterns are binary16 instead of bfloat16
 cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, int64_t x8_pitch, float *dx,
-                               bool operand_order, cudaStream_t st);
+                               bool operand_order, bool act_f16, cudaStream_t st);
 
 cudaError_t launch_wait_timeout(int *status, long long limit_cycles, cudaStream_t st);
 
@@ -62,7 +63,7 @@ GemvPlan gemv_plan(const Dims &d, int64_t M, int mode);
 
 // Small-M (M <= 16) split-K tensor-core GEMV, both activation modes.
 cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
-                        uint8_t *ws, const Workspace &plan, cudaStream_t st);
+                        bool act_f16, uint8_t *ws, const Workspace &plan, cudaStream_t st);
 int gemm_tc_token_tile(int64_t M);
 int gemm_tc_split_k(const Dims &d, int64_t M);
 int gemm_a8_token_tile(const Dims &d, int64_t M);
@@ -79,10 +80,10 @@ cudaError_t launch_encode_search(const float *W, int B, int G, int64_t N, int64_
                                  float *scale, uint16_t *a, uint16_t *b, cudaStream_t st);
 // Large-M tcgen05 / TMEM GEMM, both activation modes.
 cudaError_t launch_gemm_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
-                           uint8_t *ws, const Workspace &plan, cudaStream_t st);
+                           bool act_f16, uint8_t *ws, const Workspace &plan, cudaStream_t st);
 
 // Large-M Dynamic-A8 GEMM: activation quantiser, then tcgen05 kind::i8 with per-group int32 partials.
-cudaError_t launch_gemm_a8_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, uint8_t *ws,
-                              const Workspace &plan, cudaStream_t st);
+cudaError_t launch_gemm_a8_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, bool act_f16,
+                              uint8_t *ws, const Workspace &plan, cudaStream_t st);
 
 }  // namespace cq

@@ -205,14 +205,14 @@ __global__ void a8_partials_kernel(const void *__restrict__ layout, Dims d, cons
 // plain version for rows whose length or addresses do not allow 16-byte accesses
 __global__ void __launch_bounds__(256) quantize_a8_scalar_kernel(const uint16_t *__restrict__ x, int64_t M, int64_t K,
                                                          int8_t *__restrict__ x8, int64_t x8_pitch,
-                                                         float *__restrict__ dx) {
+                                                         float *__restrict__ dx, bool f16) {
     __shared__ float red[8];
     __shared__ float s_d;
     const int64_t m = blockIdx.x;
     const uint16_t *row = x + m * K;
     float mx = 0.0f;
     for (int64_t j = threadIdx.x; j < K; j += blockDim.x)
-        mx = fmaxf(mx, fabsf(__uint_as_float((uint32_t)row[j] << 16)));
+        mx = fmaxf(mx, fabsf(act_to_float(row[j], f16)));
     for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
     __syncthreads();
@@ -230,7 +230,7 @@ __global__ void __launch_bounds__(256) quantize_a8_scalar_kernel(const uint16_t 
     for (int64_t j = threadIdx.x; j < x8_pitch; j += blockDim.x) {
         int q = 0;
         if (j < K) {
-            const float v = __fdiv_rn(__uint_as_float((uint32_t)row[j] << 16), d);
+            const float v = __fdiv_rn(act_to_float(row[j], f16), d);
             float r = roundf(v);  // halves away from zero
             r = fminf(fmaxf(r, -127.0f), 127.0f);
             q = (int)r;
@@ -243,7 +243,7 @@ __global__ void __launch_bounds__(256) quantize_a8_scalar_kernel(const uint16_t 
 template <bool OPERAND_ORDER>
 __global__ void __launch_bounds__(1024) quantize_a8_kernel(const uint16_t *__restrict__ x, int64_t M, int64_t K,
                                                           int8_t *__restrict__ x8, int64_t x8_pitch,
-                                                          float *__restrict__ dx) {
+                                                          float *__restrict__ dx, bool f16) {
     // the kernel launched next may start now (its first steps do not touch what this one writes)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __shared__ unsigned red[32];
@@ -269,7 +269,7 @@ __global__ void __launch_bounds__(1024) quantize_a8_kernel(const uint16_t *__res
         unsigned v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0u;
         v = __reduce_max_sync(0xffffffffu, v);
         if (threadIdx.x == 0) {
-            const float xbar = fmaxf(__uint_as_float(v << 16), 1e-10f);
+            const float xbar = fmaxf(act_to_float(v, f16), 1e-10f);
             const float d = __fdiv_rn(xbar, 127.0f);
             s_d = d;
             dx[m] = d;
@@ -287,8 +287,8 @@ __global__ void __launch_bounds__(1024) quantize_a8_kernel(const uint16_t *__res
             const uint32_t ws[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
-                const uint32_t bits = (q & 1) ? (ws[q >> 1] & 0xFFFF0000u) : (ws[q >> 1] << 16);
-                float r = roundf(__fdiv_rn(__uint_as_float(bits), d));  // halves away from zero
+                const uint32_t bits16 = (q & 1) ? (ws[q >> 1] >> 16) : (ws[q >> 1] & 0xFFFFu);
+                float r = roundf(__fdiv_rn(act_to_float(bits16, f16), d));  // halves away from zero
                 r = fminf(fmaxf(r, -127.0f), 127.0f);
                 out[q >> 2] |= ((uint32_t)(int)r & 0xFFu) << (8 * (q & 3));
             }
@@ -359,19 +359,19 @@ cudaError_t launch_a8_partials(const void *layout, const Dims &d, const int8_t *
     return cudaGetLastError();
 }
 cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, int64_t x8_pitch, float *dx,
-                               bool operand_order, cudaStream_t st) {
+                               bool operand_order, bool act_f16, cudaStream_t st) {
     const bool wide = K % 8 == 0 && x8_pitch % 8 == 0 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0 &&
                       (reinterpret_cast<uintptr_t>(x8) & 7u) == 0;
     if (operand_order && !(wide && x8_pitch % 32 == 0)) return cudaErrorInvalidValue;   // internal callers pad the pitch to 128
     if (!wide) {
-        quantize_a8_scalar_kernel<<<(unsigned)M, 256, 0, st>>>(x, M, K, x8, x8_pitch, dx);
+        quantize_a8_scalar_kernel<<<(unsigned)M, 256, 0, st>>>(x, M, K, x8, x8_pitch, dx, act_f16);
         return cudaGetLastError();
     }
     int64_t threads = ((K >> 3) + 31) / 32 * 32;   // one 8-value chunk per thread when the row is short enough
     if (threads > 1024) threads = 1024;
     if (M > 64 && threads > 256) threads = 256;    // many rows: smaller CTAs fill the SMs better
-    if (operand_order) quantize_a8_kernel<true><<<(unsigned)M, (unsigned)threads, 0, st>>>(x, M, K, x8, x8_pitch, dx);
-    else quantize_a8_kernel<false><<<(unsigned)M, (unsigned)threads, 0, st>>>(x, M, K, x8, x8_pitch, dx);
+    if (operand_order) quantize_a8_kernel<true><<<(unsigned)M, (unsigned)threads, 0, st>>>(x, M, K, x8, x8_pitch, dx, act_f16);
+    else quantize_a8_kernel<false><<<(unsigned)M, (unsigned)threads, 0, st>>>(x, M, K, x8, x8_pitch, dx, act_f16);
     return cudaGetLastError();
 }
 

@@ -66,7 +66,7 @@ extern "C" int cq_gemv_static(const void *layout, int B, int G, const uint16_t *
     if (e != cudaSuccess) return cuda_failed(e);
     e = cudaMemsetAsync(ws + plan.counters_off, 0, plan.counters_bytes, st);
     if (e != cudaSuccess) return cuda_failed(e);
-    e = launch_gemv(layout, d, x, y, M, CQ_MODEL_DTYPE, ws, plan, st);
+    e = launch_gemv(layout, d, x, y, M, CQ_MODEL_DTYPE, false, ws, plan, st);
     return e == cudaSuccess ? CQ_OK : cuda_failed(e);
 }
 #pragma GCC visibility pop

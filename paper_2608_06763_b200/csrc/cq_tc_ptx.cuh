@@ -108,6 +108,10 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
 __host__ __device__ constexpr uint32_t idesc_bf16(int BN) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
+// The same with A and B binary16 (format code 0 in both operand fields).
+__host__ __device__ constexpr uint32_t idesc_f16(int BN) {
+    return (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
 
 
 // D[tmem] (+)= A[smem desc] * B[smem desc], int8 inputs, int32 accumulate

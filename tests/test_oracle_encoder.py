@@ -216,3 +216,15 @@ def test_model_product_matches_dense_matmul():
     # reconstruction is close to the source weights (NRMSE at W4 on Laplace groups ~ 0.1)
     nrmse = math.sqrt(((W - What) ** 2).sum() / (W.astype(np.float64) ** 2).sum())
     assert nrmse < 0.16
+    # binary16 activations (Section 5.3: the model-dtype path accepts FP16 or BF16): the same dense matmul on the
+    # values numpy's float16 gives those bit patterns; and on values both formats hold exactly the two dtypes agree
+    xh = datagen.bf16_bits_to_f32(x).astype(np.float16)
+    yh = oracle.gemm_model(codes, s, a, b, B, G, K, xh.view(np.uint16), act="f16")
+    assert np.allclose(yh, xh.astype(np.float64) @ What.T, rtol=1e-13, atol=1e-18)
+    small = np.round(datagen.bf16_bits_to_f32(x) * 8.0) / 8.0            # multiples of 1/8 below 32: exact in bf16 and fp16
+    yb = oracle.gemm_model(codes, s, a, b, B, G, K, datagen.to_bf16_bits(small))
+    yf = oracle.gemm_model(codes, s, a, b, B, G, K, small.astype(np.float16).view(np.uint16), act="f16")
+    assert np.array_equal(yb, yf)
+    x8b, dxb = oracle.quantize_a8(datagen.to_bf16_bits(small))
+    x8f, dxf = oracle.quantize_a8(small.astype(np.float16).view(np.uint16), act="f16")
+    assert np.array_equal(x8b, x8f) and np.array_equal(dxb, dxf)
