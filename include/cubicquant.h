@@ -100,6 +100,25 @@ int cq_gemm(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, in
 int cq_gemm_f16(const void *layout, int B, int G, const uint16_t *x, uint16_t *y, int64_t M, int64_t N, int64_t K,
                 int mode, void *workspace, size_t workspace_bytes, void *stream);
 
+/* A SwiGLU MLP block with the boundary in front of the down projection fused (Section 5.4, last paragraph:
+ * activation and quantisation combined adjacent to the down projection; Section 6.4 says where the boundary must
+ * not sit: the intermediate only changes its global-memory dtype if it is written out as a carrier by the
+ * producing GEMM).  Three launches:
+ *     h   = gate_up(x)                          [M][2 I], model dtype; gate = h[:, :I], up = h[:, I:]
+ *     act = silu(gate) * up, rounded to the model dtype, and at once its Dynamic-A8 carrier and row scales
+ *           (one kernel; the activation itself never reaches memory)
+ *     y   = down(act) in Dynamic A8             [M][N], model dtype
+ * so the result equals cq_gemm(gate_up) -> an elementwise activation operator -> cq_gemm(down, CQ_DYN_A8).
+ * layout_gate_up: device layout of the 2 I x K matrix; layout_down: of the N x I matrix; x [M][K], y [M][N];
+ * mode_gate_up: CQ_MODEL_DTYPE or CQ_DYN_A8; act_f16: 0 = bfloat16, 1 = binary16 activations and output.
+ * workspace: cq_mlp_workspace_bytes() bytes, zeroed once with cq_workspace_init; cq_gemm_status(workspace) reports a
+ * bounded wait of either projection that gave up.  Errors as cq_gemm; I must be a multiple of 8. */
+size_t cq_mlp_workspace_bytes(int B_gate_up, int G_gate_up, int B_down, int G_down, int64_t M, int64_t K, int64_t I, int64_t N,
+                              int mode_gate_up);
+int cq_mlp_swiglu(const void *layout_gate_up, int B_gate_up, int G_gate_up, const void *layout_down, int B_down, int G_down,
+                  const uint16_t *x, uint16_t *y, int64_t M, int64_t K, int64_t I, int64_t N, int mode_gate_up, int act_f16,
+                  void *workspace, size_t workspace_bytes, void *stream);
+
 /* Reads back the device status word of a workspace (waits for `stream` first).  CQ_OK, or
  * CQ_ERR_TIMEOUT when a bounded device-side wait of an earlier cq_gemm on this workspace gave up
  * (its output is then undefined; re-initialise the workspace before reusing it). */

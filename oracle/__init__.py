@@ -295,3 +295,42 @@ def gemm_a8(codes, s, a, b, B, G, K, x8, dx, rows=None, cols=None, want_partials
                             _p(x8), _p(dx), C.c_int64(M), _p(r), C.c_int64(nr), _p(c), C.c_int64(nc), _p(y), _p(P))
     assert bad == 0, "int32 partial bound |P_g| <= G*127^2 violated"
     return (y, P) if want_partials else y
+
+
+# ----------------------------------------------------------------------------- fused MLP boundary
+def silu_mul(gate: np.ndarray, up: np.ndarray) -> np.ndarray:
+    """The gated activation of a SwiGLU MLP in fp64: silu(gate) * up, silu(g) = g / (1 + exp(-g))."""
+    g = np.asarray(gate, np.float64)
+    return g / (1.0 + np.exp(-g)) * np.asarray(up, np.float64)
+
+
+def _to_bf16_bits(v: np.ndarray) -> np.ndarray:
+    """fp64 -> bfloat16 bit patterns, round to nearest even (through fp32, which holds every bf16 midpoint)."""
+    f = np.ascontiguousarray(v, dtype=np.float32)
+    u = f.view(np.uint32)
+    return ((u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)).astype(np.uint16)
+
+
+def mlp_swiglu(gate_up, down, x_bf16, mode_gate_up: str = "model"):
+    """The MLP boundary of Section 5.4 (last paragraph: activation and quantisation fused next to the down
+    projection) as the plain composition of the operators it fuses, each with its operator-local semantics:
+
+        h   = gate_up(x)                 model dtype or Dynamic A8, output rounded to the model dtype (bf16)
+        act = bf16(silu(h[:, :I]) * h[:, I:])
+        y   = down(act) in Dynamic A8    per-row absmax INT8 of act, INT8 carriers, int32 partials, fp32 rescale
+
+    gate_up / down: dicts with codes, s, a, b, B, G, K (gate_up has 2 I output channels, down has K = I).
+    Returns (y fp64 [M, N], act bf16 bits [M, I])."""
+    gu, dn = gate_up, down
+    if mode_gate_up == "model":
+        h = gemm_model(gu["codes"], gu["s"], gu["a"], gu["b"], gu["B"], gu["G"], gu["K"], x_bf16)
+    else:
+        x8, dx = quantize_a8(x_bf16)
+        h = gemm_a8(gu["codes"], gu["s"], gu["a"], gu["b"], gu["B"], gu["G"], gu["K"], x8, dx)
+    hb = _to_bf16_bits(h)
+    hv = (hb.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    inter = hv.shape[1] // 2
+    act = _to_bf16_bits(silu_mul(hv[:, :inter], hv[:, inter:]))
+    a8, da = quantize_a8(act)
+    y = gemm_a8(dn["codes"], dn["s"], dn["a"], dn["b"], dn["B"], dn["G"], dn["K"], a8, da)
+    return y, act

@@ -51,6 +51,10 @@ def lib():
         L.cq_gemm.argtypes = [vp, i, i, vp, vp, i64, i64, i64, i, vp, sz, vp]
         L.cq_gemm_f16.argtypes = [vp, i, i, vp, vp, i64, i64, i64, i, vp, sz, vp]
         L.cq_quantize_a8_f16.argtypes = [vp, i64, i64, vp, vp, vp]
+        L.cq_mlp_workspace_bytes.restype = sz
+        L.cq_mlp_workspace_bytes.argtypes = [i, i, i, i, i64, i64, i64, i64, i]
+        L.cq_mlp_swiglu.argtypes = [vp, i, i, vp, i, i, vp, vp, i64, i64, i64, i64, i, i, vp, sz, vp]
+        L.cq_mlp_swiglu.restype = i
         L.cq_gemm_status.argtypes = [vp, sz, vp]
         L.cq_gemm_status.restype = i
         L.cq_gemv_static.argtypes = [vp, i, i, vp, vp, i64, i64, i64, vp]
@@ -168,6 +172,23 @@ def cq_gemm(pw: PackedWeights, x: torch.Tensor, mode: int = CQ_MODEL_DTYPE, work
     fn = lib().cq_gemm if x.dtype == torch.bfloat16 else lib().cq_gemm_f16
     _check(fn(_ptr(pw.layout), pw.B, pw.G, _ptr(x), _ptr(y), M, pw.N, pw.K, mode, _ptr(workspace),
                          workspace.numel(), _stream()), "cq_gemm")
+    return y
+
+
+def cq_mlp_swiglu(gate_up: PackedWeights, down: PackedWeights, x: torch.Tensor, mode_gate_up: int = CQ_MODEL_DTYPE,
+                  workspace: torch.Tensor | None = None, out: torch.Tensor | None = None) -> torch.Tensor:
+    """y[M, N] = down(silu(gate) * up) with (gate | up) = gate_up(x): the SwiGLU MLP block whose activation and
+    Dynamic-A8 quantiser in front of the down projection are one kernel.  gate_up is 2 I x K, down is N x I."""
+    assert x.dtype in (torch.bfloat16, torch.float16) and x.dim() == 2 and x.shape[1] == gate_up.K
+    M, K, I, N = x.shape[0], gate_up.K, down.K, down.N
+    assert gate_up.N == 2 * I
+    need = lib().cq_mlp_workspace_bytes(gate_up.B, gate_up.G, down.B, down.G, M, K, I, N, mode_gate_up)
+    if workspace is None:
+        workspace = torch.zeros(need, dtype=torch.uint8, device=x.device)
+    y = out if out is not None else torch.empty((M, N), dtype=x.dtype, device=x.device)
+    _check(lib().cq_mlp_swiglu(_ptr(gate_up.layout), gate_up.B, gate_up.G, _ptr(down.layout), down.B, down.G, _ptr(x), _ptr(y),
+                               M, K, I, N, mode_gate_up, 1 if x.dtype == torch.float16 else 0, _ptr(workspace),
+                               workspace.numel(), _stream()), "cq_mlp_swiglu")
     return y
 
 

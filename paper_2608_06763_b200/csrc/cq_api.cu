@@ -166,6 +166,64 @@ int cq_gemm_f16(const void *layout, int B, int G, const uint16_t *x, uint16_t *y
     return gemm_any(layout, B, G, x, y, M, N, K, mode, true, workspace, workspace_bytes, stream);
 }
 
+// Workspace of the fused MLP: [gate_up operator's workspace][h: M x 2 I model-dtype values][down operator's
+// Dynamic-A8 workspace].  The down operator's plan is shifted so that both operators report into the one status
+// word at the front.
+struct MlpPlan { Workspace gu, dn; size_t h_off, total; };
+static MlpPlan plan_mlp(const Dims &dgu, const Dims &ddn, int64_t M, int mode_gu) {
+    MlpPlan p;
+    p.gu = plan_workspace(dgu, M, mode_gu);
+    p.h_off = align_up(p.gu.total, 256);
+    const size_t dn_off = align_up(p.h_off + (size_t)M * (size_t)dgu.N * 2, 256);
+    p.dn = plan_workspace(ddn, M, CQ_DYN_A8);
+    p.dn.counters_off += dn_off; p.dn.partial_off += dn_off; p.dn.x8_off += dn_off; p.dn.dx_off += dn_off;
+    p.dn.status_off = 0;
+    p.total = dn_off + p.dn.total;
+    return p;
+}
+
+size_t cq_mlp_workspace_bytes(int B_gu, int G_gu, int B_dn, int G_dn, int64_t M, int64_t K, int64_t I, int64_t N, int mode_gate_up) {
+    if (check_format(B_gu, G_gu, 2 * I, K) != CQ_OK || check_format(B_dn, G_dn, N, I) != CQ_OK || M <= 0) return 0;
+    if (mode_gate_up != CQ_MODEL_DTYPE && mode_gate_up != CQ_DYN_A8) return 0;
+    return plan_mlp(make_dims(B_gu, G_gu, 2 * I, K), make_dims(B_dn, G_dn, N, I), M, mode_gate_up).total;
+}
+
+int cq_mlp_swiglu(const void *layout_gate_up, int B_gu, int G_gu, const void *layout_down, int B_dn, int G_dn, const uint16_t *x,
+                  uint16_t *y, int64_t M, int64_t K, int64_t I, int64_t N, int mode_gate_up, int act_f16, void *workspace,
+                  size_t workspace_bytes, void *stream) {
+    if (!layout_gate_up || !layout_down || !x || !y || !workspace || M <= 0 || I <= 0) return CQ_ERR_INVALID_ARG;
+    if (mode_gate_up != CQ_MODEL_DTYPE && mode_gate_up != CQ_DYN_A8) return CQ_ERR_INVALID_ARG;
+    int st = check_format(B_gu, G_gu, 2 * I, K);
+    if (st == CQ_OK) st = check_format(B_dn, G_dn, N, I);
+    if (st != CQ_OK) return st;
+    if (I % 8 != 0) return CQ_ERR_UNSUPPORTED;
+    if (misaligned(layout_gate_up) || misaligned(layout_down) || misaligned(x) || misaligned(y) || misaligned(workspace))
+        return CQ_ERR_ALIGNMENT;
+    const Dims dgu = make_dims(B_gu, G_gu, 2 * I, K), ddn = make_dims(B_dn, G_dn, N, I);
+    const MlpPlan plan = plan_mlp(dgu, ddn, M, mode_gate_up);
+    if (workspace_bytes < plan.total) return CQ_ERR_WORKSPACE;
+    st = check_arch();
+    if (st != CQ_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    uint8_t *ws = (uint8_t *)workspace;
+    uint16_t *h = reinterpret_cast<uint16_t *>(ws + plan.h_off);
+    const bool f16 = act_f16 != 0;
+    // 1. gate_up, an ordinary operator: model-dtype output
+    cudaError_t e;
+    if (M <= 16) e = launch_gemv(layout_gate_up, dgu, x, h, M, mode_gate_up, f16, ws, plan.gu, s);
+    else if (mode_gate_up == CQ_MODEL_DTYPE) e = launch_gemm_tc(layout_gate_up, dgu, x, h, M, mode_gate_up, f16, ws, plan.gu, s);
+    else e = launch_gemm_a8_tc(layout_gate_up, dgu, x, h, M, f16, ws, plan.gu, s);
+    if (e != cudaSuccess) return wrap(e);
+    // 2. gated activation and the down projection's activation quantiser in one kernel
+    e = launch_swiglu_quantize_a8(h, M, I, reinterpret_cast<int8_t *>(ws + plan.dn.x8_off), (int64_t)ddn.KT * TILE,
+                                  reinterpret_cast<float *>(ws + plan.dn.dx_off), f16, s);
+    if (e != cudaSuccess) return wrap(e);
+    // 3. the down projection on the carrier that is already in its workspace
+    if (M <= 16) e = launch_gemv(layout_down, ddn, nullptr, y, M, CQ_DYN_A8, f16, ws, plan.dn, s, true);
+    else e = launch_gemm_a8_tc(layout_down, ddn, nullptr, y, M, f16, ws, plan.dn, s, true);
+    return wrap(e);
+}
+
 int cq_gemm_status(const void *workspace, size_t workspace_bytes, void *stream) {
     if (!workspace || workspace_bytes < 512) return CQ_ERR_INVALID_ARG;
     // the status word is the first word of every workspace (plan_workspace)

@@ -411,15 +411,17 @@ cudaError_t launch_a8_b(const void *layout, const Dims &d, const int8_t *x8, int
 
 // Quantise the activations (one block per row), then run the tcgen05 INT8 GEMM on the carriers.
 cudaError_t launch_gemm_a8_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, bool act_f16,
-                              uint8_t *ws, const Workspace &plan, cudaStream_t st) {
+                              uint8_t *ws, const Workspace &plan, cudaStream_t st, bool prequantized) {
     int8_t *xq = reinterpret_cast<int8_t *>(ws + plan.x8_off);
     float *dxs = reinterpret_cast<float *>(ws + plan.dx_off);
     int *status = reinterpret_cast<int *>(ws + plan.status_off);
     float *partial = reinterpret_cast<float *>(ws + plan.partial_off);
     int *counters = reinterpret_cast<int *>(ws + plan.counters_off);
     const int64_t pitch = (int64_t)d.KT * TILE;
-    cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, true, act_f16, st);
-    if (e != cudaSuccess) return e;
+    if (!prequantized) {
+        cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, true, act_f16, st);
+        if (e != cudaSuccess) return e;
+    }
     switch (d.B) {
         case 1: return launch_a8_b<1>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, act_f16, st);
         case 2: return launch_a8_b<2>(layout, d, xq, pitch, dxs, y, M, status, partial, counters, act_f16, st);

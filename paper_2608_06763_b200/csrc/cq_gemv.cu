@@ -963,7 +963,7 @@ GemvPlan gemv_plan(const Dims &d, int64_t M, int mode) {
 }
 
 cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
-                        bool act_f16, uint8_t *ws, const Workspace &plan, cudaStream_t st) {
+                        bool act_f16, uint8_t *ws, const Workspace &plan, cudaStream_t st, bool prequantized) {
     const GemvPlan gp = gemv_plan(d, M, mode);
     float *partial = reinterpret_cast<float *>(ws + plan.partial_off);
     int *counters = reinterpret_cast<int *>(ws + plan.counters_off);
@@ -971,7 +971,7 @@ cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, ui
     int8_t *xq = reinterpret_cast<int8_t *>(ws + plan.x8_off);
     float *dxs = reinterpret_cast<float *>(ws + plan.dx_off);
     const int64_t pitch = (int64_t)d.KT * TILE;
-    if (mode == 1) {
+    if (mode == 1 && !prequantized) {
         cudaError_t e = launch_quantize_a8(x, M, d.K, xq, pitch, dxs, true, act_f16, st);
         if (e != cudaSuccess) return e;
     }

@@ -22,6 +22,9 @@ cudaError_t launch_a8_partials(const void *layout, const Dims &d, const int8_t *
 cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *x8, int64_t x8_pitch, float *dx,
                                bool operand_order, bool act_f16, cudaStream_t st);
 
+// h[M][2 I] (gate | up, model dtype) -> INT8 carrier of silu(gate) * up in the MMA operand order, and its row scales
+cudaError_t launch_swiglu_quantize_a8(const uint16_t *h, int64_t M, int64_t I, int8_t *x8, int64_t x8_pitch, float *dx,
+                                      bool act_f16, cudaStream_t st);
 cudaError_t launch_wait_timeout(int *status, long long limit_cycles, cudaStream_t st);
 
 // Workspace carving (all offsets 256-byte aligned).
@@ -62,8 +65,9 @@ struct GemvPlan { int ctas, max_run, overhead; };
 GemvPlan gemv_plan(const Dims &d, int64_t M, int mode);
 
 // Small-M (M <= 16) split-K tensor-core GEMV, both activation modes.
+// prequantized (Dynamic A8 only): the workspace already holds the INT8 carrier and the row scales of x (x is not read)
 cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
-                        bool act_f16, uint8_t *ws, const Workspace &plan, cudaStream_t st);
+                        bool act_f16, uint8_t *ws, const Workspace &plan, cudaStream_t st, bool prequantized = false);
 int gemm_tc_token_tile(int64_t M);
 int gemm_tc_split_k(const Dims &d, int64_t M);
 int gemm_a8_token_tile(const Dims &d, int64_t M);
@@ -84,6 +88,6 @@ cudaError_t launch_gemm_tc(const void *layout, const Dims &d, const uint16_t *x,
 
 // Large-M Dynamic-A8 GEMM: activation quantiser, then tcgen05 kind::i8 with per-group int32 partials.
 cudaError_t launch_gemm_a8_tc(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, bool act_f16,
-                              uint8_t *ws, const Workspace &plan, cudaStream_t st);
+                              uint8_t *ws, const Workspace &plan, cudaStream_t st, bool prequantized = false);
 
 }  // namespace cq

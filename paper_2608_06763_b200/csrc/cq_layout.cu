@@ -309,6 +309,84 @@ __global__ void __launch_bounds__(1024) quantize_a8_kernel(const uint16_t *__res
     }
 }
 
+// ---------------------------------------------------------------- fused gated activation + quantiser
+// The boundary in front of an MLP's down projection (Section 5.4, last paragraph): the row of the gate_up
+// output h[m] = (gate | up), 2 I values in the model dtype, goes to act = silu(gate) * up -- evaluated in fp32
+// and rounded to the model dtype, which is what a separate activation operator would have written -- and
+// straight on to that row's Dynamic-A8 carrier (Eq. a8-activation-scale, Eq. a8-activation-quantization) in the
+// MMA operand order, without the activation ever reaching memory.  One CTA per row; I % 8 == 0.
+__device__ __forceinline__ uint32_t gated_act_bits(uint32_t g16, uint32_t u16, bool f16) {
+    const float g = act_to_float(g16, f16), u = act_to_float(u16, f16);
+    const float sg = __fdiv_rn(g, __fadd_rn(1.0f, expf(-g)));
+    return float_to_act(__fmul_rn(sg, u), f16);
+}
+__device__ __forceinline__ uint4 gated_act_chunk(const uint4 &g, const uint4 &u, bool f16) {
+    const uint32_t gw[4] = {g.x, g.y, g.z, g.w}, uw[4] = {u.x, u.y, u.z, u.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+        o[q] = gated_act_bits(gw[q] & 0xFFFFu, uw[q] & 0xFFFFu, f16) | (gated_act_bits(gw[q] >> 16, uw[q] >> 16, f16) << 16);
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+__global__ void __launch_bounds__(1024) swiglu_quantize_a8_kernel(const uint16_t *__restrict__ h, int64_t M, int64_t I,
+                                                                 int8_t *__restrict__ x8, int64_t x8_pitch,
+                                                                 float *__restrict__ dx, bool f16) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");               // h comes from the kernel launched before
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    __shared__ unsigned red[32];
+    __shared__ float s_d;
+    const int64_t m = blockIdx.x;
+    const uint4 *grow = reinterpret_cast<const uint4 *>(h + m * 2 * I), *urow = reinterpret_cast<const uint4 *>(h + m * 2 * I + I);
+    const int64_t chunks = I >> 3;
+    uint4 keep = make_uint4(0, 0, 0, 0);   // this thread's first chunk of the activation stays in registers
+    unsigned mx = 0;
+    for (int64_t j = threadIdx.x; j < chunks; j += blockDim.x) {
+        const uint4 v = gated_act_chunk(grow[j], urow[j], f16);
+        if (j == threadIdx.x) keep = v;
+        const uint32_t ws[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { mx = max(mx, ws[q] & 0x7FFFu); mx = max(mx, (ws[q] >> 16) & 0x7FFFu); }
+    }
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        unsigned v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0u;
+        v = __reduce_max_sync(0xffffffffu, v);
+        if (threadIdx.x == 0) {
+            const float xbar = fmaxf(act_to_float(v, f16), 1e-10f);
+            const float d = __fdiv_rn(xbar, 127.0f);
+            s_d = d;
+            dx[m] = d;
+        }
+    }
+    __syncthreads();
+    const float d = s_d;
+    const int64_t out_chunks = x8_pitch >> 3;
+    for (int64_t j = threadIdx.x; j < out_chunks; j += blockDim.x) {
+        uint32_t out[2] = {0u, 0u};
+        if (j < chunks) {
+            const uint4 v = (j == threadIdx.x) ? keep : gated_act_chunk(grow[j], urow[j], f16);
+            const uint32_t ws[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const uint32_t bits16 = (q & 1) ? (ws[q >> 1] >> 16) : (ws[q >> 1] & 0xFFFFu);
+                float r = roundf(__fdiv_rn(act_to_float(bits16, f16), d));
+                r = fminf(fmaxf(r, -127.0f), 127.0f);
+                out[q >> 2] |= ((uint32_t)(int)r & 0xFFu) << (8 * (q & 3));
+            }
+        }
+        // the operand order of quantize_a8_kernel<true>
+        uint8_t *blk = reinterpret_cast<uint8_t *>(x8 + m * x8_pitch) + (j >> 2) * 32 + 2 * ((j >> 1) & 1) + 16 * (j & 1);
+#pragma unroll
+        for (int tt = 0; tt < 2; ++tt) {
+            const uint32_t pr = __byte_perm(out[tt], 0u, 0x3120);
+            *reinterpret_cast<uint16_t *>(blk + 8 * tt) = (uint16_t)pr;
+            *reinterpret_cast<uint16_t *>(blk + 8 * tt + 4) = (uint16_t)(pr >> 16);
+        }
+    }
+}
+
 // ---------------------------------------------------------------- launchers
 static inline unsigned blocks_for(int64_t n, int t) { return (unsigned)((n + t - 1) / t); }
 
@@ -373,6 +451,24 @@ cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *
     if (operand_order) quantize_a8_kernel<true><<<(unsigned)M, (unsigned)threads, 0, st>>>(x, M, K, x8, x8_pitch, dx, act_f16);
     else quantize_a8_kernel<false><<<(unsigned)M, (unsigned)threads, 0, st>>>(x, M, K, x8, x8_pitch, dx, act_f16);
     return cudaGetLastError();
+}
+
+cudaError_t launch_swiglu_quantize_a8(const uint16_t *h, int64_t M, int64_t I, int8_t *x8, int64_t x8_pitch, float *dx,
+                                      bool act_f16, cudaStream_t st) {
+    if (I % 8 != 0 || x8_pitch % 32 != 0 || (reinterpret_cast<uintptr_t>(h) & 15u) != 0) return cudaErrorInvalidValue;
+    int64_t threads = ((I >> 3) + 31) / 32 * 32;
+    if (threads > 1024) threads = 1024;
+    if (M > 64 && threads > 256) threads = 256;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)M);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, swiglu_quantize_a8_kernel, h, M, I, x8, x8_pitch, dx, act_f16);
 }
 
 // ---------------------------------------------------------------- cq_debug_wait_timeout
