@@ -286,6 +286,35 @@ def extra_suites(torch, cq, datagen, stream, peaks):
                               "us_a8": round(t[1] * 1e3, 2), "model_over_a8": round(t[0] / t[1], 3)})
         del copies
         torch.cuda.empty_cache()
+    # ---- fused MLP boundary (Section 5.4, last paragraph) on the Llama-3-8B MLP: gate_up 4096 -> 2 x 14336, down
+    # 14336 -> 4096, W4 G128; gate_up in model dtype, down in Dynamic A8; against the same chain with a separate
+    # elementwise activation operator (torch) and the down projection quantising its own input
+    mlp = []
+    K, I, N = 4096, 14336, 4096
+    Wgu = datagen.weights_cuda("outlier", 2 * I, K, seed=6, sigma=0.02, sigma_out=0.2, p=0.001)
+    Wdn = datagen.weights_cuda("outlier", N, I, seed=7, sigma=0.02, sigma_out=0.2, p=0.001)
+    pgu, pdn = fit_pack(cq, Wgu, 4, 128), fit_pack(cq, Wdn, 4, 128)
+    del Wgu, Wdn
+    for M in (1, 16, 256, 1024):
+        x = datagen.activations_cuda(M, K, seed=6)
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        h = torch.empty((M, 2 * I), dtype=torch.bfloat16, device="cuda")
+        wsm = torch.zeros(cq.lib().cq_mlp_workspace_bytes(4, 128, 4, 128, M, K, I, N, 0), dtype=torch.uint8, device="cuda")
+        ws1 = torch.zeros(cq.cq_workspace_bytes(4, 128, M, 2 * I, K, 0), dtype=torch.uint8, device="cuda")
+        ws2 = torch.zeros(cq.cq_workspace_bytes(4, 128, M, N, I, 1), dtype=torch.uint8, device="cuda")
+        fused = lambda i: cq.cq_mlp_swiglu(pgu, pdn, x, cq.CQ_MODEL_DTYPE, wsm, y)
+
+        def chain(i):
+            cq.cq_gemm(pgu, x, cq.CQ_MODEL_DTYPE, ws1, h)
+            act = torch.nn.functional.silu(h[:, :I]) * h[:, I:]
+            cq.cq_gemm(pdn, act, cq.CQ_DYN_A8, ws2, y)
+        fused(0); chain(0)
+        tf, tc = time_graph(torch, stream, fused, 8), time_graph(torch, stream, chain, 8)
+        mlp.append({"M": M, "us_fused": round(tf * 1e3, 2), "us_operator_by_operator": round(tc * 1e3, 2),
+                    "speedup": round(tc / tf, 3)})
+    out["mlp_fused_boundary_llama8b_w4g128"] = mlp
+    del pgu, pdn
+    torch.cuda.empty_cache()
     # ---- the paper's own kernel-measurement shapes (Section 6.3: G512, W2/W5/W8, M in {1,16,64,256}),
     # so B200 numbers can sit beside its H200 table (context only)
     paper = []

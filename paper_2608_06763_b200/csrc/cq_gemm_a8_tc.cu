@@ -107,6 +107,8 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
         for (int s = 0; s < A8_RAW_STAGES; ++s) { mbar_init(&raw_full[s], 1); mbar_init(&raw_empty[s], A8_WORK_WARPS); }
         for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], A8_WORK_WARPS); }
         fence_barrier_init();
+        tmem_slot[2] = 0;   // the work warps' "a wait gave up" flag
+        tmem_slot[3] = prm.f16 ? 1u : 0u;   // the output dtype, parked in shared memory: a register held across the main loop is one too many
     }
     if (threadIdx.x < 128) sT[threadIdx.x] = __fdiv_rn((float)threadIdx.x, (float)Mx);  // the pinned t = i / M
     if (warp == 1) {
@@ -171,18 +173,13 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
         // its partner of the row block would then wait for it at the 64-thread barrier for ever.  The warp
         // keeps walking the blocks instead, without waiting any more, so every barrier still sees both
         // warps; what it computes from then on is discarded (the status word is set, nothing is stored).
-        bool ok = true;
-        auto wait_or_give_up = [&](uint64_t *bar, uint32_t parity, int code) {
-            if (!ok) return;
-            const bool flipped = mbar_wait(bar, parity, prm.status, code);
-            ok = !__any_sync(0xffffffffu, !flipped);   // the warp decides as one
-        };
+        volatile int *gave_up = reinterpret_cast<volatile int *>(tmem_slot + 2);   // CTA-wide flag, cleared at start
         for (int t = 0; t <= KT; ++t) {
             if (t < KT) {
                 // ---------------- (a) decode block t
                 const int rs = t % A8_RAW_STAGES, s = t % A8_STAGES;
-                wait_or_give_up(&raw_full[rs], (t / A8_RAW_STAGES) & 1, 16);
-                if (t >= A8_STAGES) wait_or_give_up(&st_empty[s], ((t / A8_STAGES) - 1) & 1, 17);
+                if (!*gave_up && !mbar_wait(&raw_full[rs], (t / A8_RAW_STAGES) & 1, prm.status, 16)) *gave_up = 1;
+                if (t >= A8_STAGES && !*gave_up && !mbar_wait(&st_empty[s], ((t / A8_STAGES) - 1) & 1, prm.status, 17)) *gave_up = 1;
                 const uint8_t *raw = sRaw + rs * prm.raw_stage_bytes;
                 const uint8_t *rbp = raw + rb * 256 * B;
                 uint32_t w[2 * B];
@@ -275,7 +272,7 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
             if (t >= 1) {
                 // ---------------- (b) drain block t - 1
                 const int td = t - 1, ab = td & 1;
-                wait_or_give_up(&acc_full[ab], (td >> 1) & 1, 18);
+                if (!*gave_up && !mbar_wait(&acc_full[ab], (td >> 1) & 1, prm.status, 18)) *gave_up = 1;
                 tc_fence_after();
                 const float *scd = sScale + (size_t)(td % A8_SRING) * 128 * GPT + drow * GPT;
 #pragma unroll
@@ -295,21 +292,27 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
                 if (lane == 0) mbar_arrive(&acc_empty[ab]);
             }
         }
-        if (ok) {
+        if (!*gave_up) {
             const int64_t n = (int64_t)nb * TILE + drow;
             if (n < d.N || gridDim.z > 1) {   // partial sums of padding channels are written too (zeros), never read back as y
+                // the output dtype is decided once, outside the loop over the 64 accumulators (a select inside it
+                // costs the registers this kernel does not have)
+                auto store_all = [&](auto f16c) {
+                    constexpr bool F16 = decltype(f16c)::value;
 #pragma unroll
-                for (int i = 0; i < QCOLS; ++i) {
-                    const int64_t m = (int64_t)mt * BN + cq4 * QCOLS + i;
-                    if (m < prm.M) {
-                        if (gridDim.z == 1) {
-                            const float v = acc[i] * (prm.dx[m] * (1.0f / 127.0f));
-                            prm.y[m * d.N + n] = float_to_act(v, prm.f16);
-                        } else {
-                            prm.partial[((size_t)blockIdx.z * prm.M + m) * ((size_t)d.NB * TILE) + n] = acc[i];
+                    for (int i = 0; i < QCOLS; ++i) {
+                        const int64_t m = (int64_t)mt * BN + cq4 * QCOLS + i;
+                        if (m < prm.M) {
+                            if (gridDim.z == 1) {
+                                const float v = acc[i] * (prm.dx[m] * (1.0f / 127.0f));
+                                prm.y[m * d.N + n] = float_to_act(v, F16);
+                            } else {
+                                prm.partial[((size_t)blockIdx.z * prm.M + m) * ((size_t)d.NB * TILE) + n] = acc[i];
+                            }
                         }
                     }
-                }
+                };
+                if (*reinterpret_cast<volatile uint32_t *>(tmem_slot + 3)) store_all(std::true_type{}); else store_all(std::false_type{});
             }
         }
     }
@@ -333,6 +336,7 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
         __syncthreads();
         if (*s_last_p) {
             const size_t Np = (size_t)d.NB * TILE;
+            const bool out_f16 = *reinterpret_cast<volatile uint32_t *>(tmem_slot + 3) != 0;
             constexpr int QUADS = BN * TILE / 4;   // four consecutive channels of one token per 128-bit load
             for (int qd = threadIdx.x; qd < QUADS; qd += A8_THREADS) {
                 const int64_t m = (int64_t)mt * BN + qd / (TILE / 4), n = (int64_t)nb * TILE + (qd % (TILE / 4)) * 4;
@@ -349,7 +353,7 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
                 const float o[4] = {sum.x * f, sum.y * f, sum.z * f, sum.w * f};
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                    if (n + e < d.N) prm.y[m * d.N + n + e] = float_to_act(o[e], prm.f16);
+                    if (n + e < d.N) prm.y[m * d.N + n + e] = float_to_act(o[e], out_f16);
             }
             if (threadIdx.x == 0) *ctr = 0;  // leave the workspace ready for the next call
         }
