@@ -30,7 +30,7 @@ int gemm_tc_token_tile(int64_t M) { return M <= 32 ? 32 : M <= 64 ? 64 : M <= 12
 int gemm_tc_split_k(const Dims &d, int64_t M) {
     const int64_t bnt = gemm_tc_token_tile(M);
     const int64_t ctas = (int64_t)d.NB * ((M + bnt - 1) / bnt);
-    if (ctas >= 100 || M > 256) return 1;   // the combine of a large token tile costs more than the idle SMs
+    if (ctas >= 100 || M > 1024) return 1;   // beyond that the output tiles alone fill the SMs, or the combine costs more than it saves
     int64_t sk = sm_count() / ctas;
     if (sk > 8) sk = 8;
     if (sk > d.KT / 4) sk = d.KT / 4;   // at least four layout tiles per slice
