@@ -119,6 +119,22 @@ int cq_mlp_swiglu(const void *layout_gate_up, int B_gate_up, int G_gate_up, cons
                   const uint16_t *x, uint16_t *y, int64_t M, int64_t K, int64_t I, int64_t N, int mode_gate_up, int act_f16,
                   void *workspace, size_t workspace_bytes, void *stream);
 
+/* Routed execution (Section 5.5): R token-matrix routes over E matrices of one shape and format, compacted and
+ * grouped by matrix so that every decoded weight tile serves all routes of its matrix.  The caller supplies the route map
+ * (routing probabilities, selection and route weights stay outside, as the paper leaves them):
+ *     layouts_host        HOST array of E device pointers (device layouts of the E matrices, each N x K)
+ *     route_token         DEVICE int32 [R]: the token (row of x) of each route, routes of matrix e at
+ *                         [expert_offset[e], expert_offset[e+1])
+ *     expert_offset_host  HOST int64 [E + 1], non-decreasing, [0] = 0, [E] = R
+ *     x [T][K], y_routes [R][N] (route-major output, model dtype); act_f16 as for cq_mlp_swiglu
+ * One gather kernel, then one ordinary cq_gemm dispatch per matrix that has routes, on `stream`.  A token index outside
+ * [0, T) yields a zero input row.  workspace: cq_routed_workspace_bytes() bytes, zeroed once with cq_workspace_init.
+ * Errors as cq_gemm; CQ_ERR_INVALID_ARG for an inconsistent offset array; N and K must be multiples of 8. */
+size_t cq_routed_workspace_bytes(int B, int G, int E, const int64_t *expert_offset_host, int64_t N, int64_t K, int mode);
+int cq_gemm_routed(const void *const *layouts_host, int E, int B, int G, const uint16_t *x, const int32_t *route_token,
+                   const int64_t *expert_offset_host, uint16_t *y_routes, int64_t T, int64_t N, int64_t K, int mode, int act_f16,
+                   void *workspace, size_t workspace_bytes, void *stream);
+
 /* Reads back the device status word of a workspace (waits for `stream` first).  CQ_OK, or
  * CQ_ERR_TIMEOUT when a bounded device-side wait of an earlier cq_gemm on this workspace gave up
  * (its output is then undefined; re-initialise the workspace before reusing it). */

@@ -334,3 +334,26 @@ def mlp_swiglu(gate_up, down, x_bf16, mode_gate_up: str = "model"):
     a8, da = quantize_a8(act)
     y = gemm_a8(dn["codes"], dn["s"], dn["a"], dn["b"], dn["B"], dn["G"], dn["K"], a8, da)
     return y, act
+
+
+# ----------------------------------------------------------------------------- routed execution
+def gemm_routed(experts, x_bits, route_token, expert_offset, mode: str = "model", act: str = "bf16") -> np.ndarray:
+    """Routed product of Section 5.5 with routes grouped by matrix: route r (in the block of matrix e) is the
+    ordinary product of token route_token[r] with matrix e.  experts: list of dicts (codes, s, a, b, B, G, K);
+    returns route-major fp64 y[R, N].  Route weights and the reduction over a token's routes are not part of it."""
+    x_bits = np.asarray(x_bits, np.uint16)
+    route_token = np.asarray(route_token, np.int64)
+    R = int(expert_offset[-1])
+    N = experts[0]["codes"].shape[0]
+    y = np.zeros((R, N), np.float64)
+    for e, w in enumerate(experts):
+        r0, r1 = int(expert_offset[e]), int(expert_offset[e + 1])
+        if r1 == r0:
+            continue
+        xe = np.ascontiguousarray(x_bits[route_token[r0:r1]])
+        if mode == "model":
+            y[r0:r1] = gemm_model(w["codes"], w["s"], w["a"], w["b"], w["B"], w["G"], w["K"], xe, act=act)
+        else:
+            x8, dx = quantize_a8(xe, act=act)
+            y[r0:r1] = gemm_a8(w["codes"], w["s"], w["a"], w["b"], w["B"], w["G"], w["K"], x8, dx)
+    return y

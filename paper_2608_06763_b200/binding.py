@@ -55,6 +55,10 @@ def lib():
         L.cq_mlp_workspace_bytes.argtypes = [i, i, i, i, i64, i64, i64, i64, i]
         L.cq_mlp_swiglu.argtypes = [vp, i, i, vp, i, i, vp, vp, i64, i64, i64, i64, i, i, vp, sz, vp]
         L.cq_mlp_swiglu.restype = i
+        L.cq_routed_workspace_bytes.restype = sz
+        L.cq_routed_workspace_bytes.argtypes = [i, i, i, vp, i64, i64, i]
+        L.cq_gemm_routed.argtypes = [vp, i, i, i, vp, vp, vp, vp, i64, i64, i64, i, i, vp, sz, vp]
+        L.cq_gemm_routed.restype = i
         L.cq_gemm_status.argtypes = [vp, sz, vp]
         L.cq_gemm_status.restype = i
         L.cq_gemv_static.argtypes = [vp, i, i, vp, vp, i64, i64, i64, vp]
@@ -189,6 +193,30 @@ def cq_mlp_swiglu(gate_up: PackedWeights, down: PackedWeights, x: torch.Tensor, 
     _check(lib().cq_mlp_swiglu(_ptr(gate_up.layout), gate_up.B, gate_up.G, _ptr(down.layout), down.B, down.G, _ptr(x), _ptr(y),
                                M, K, I, N, mode_gate_up, 1 if x.dtype == torch.float16 else 0, _ptr(workspace),
                                workspace.numel(), _stream()), "cq_mlp_swiglu")
+    return y
+
+
+def cq_gemm_routed(experts, x: torch.Tensor, route_token: torch.Tensor, expert_offset, mode: int = CQ_MODEL_DTYPE,
+                   workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """Route-major y[R, N]: route r multiplies token route_token[r] of x by the matrix whose block
+    [expert_offset[e], expert_offset[e+1]) holds r.  experts: list of PackedWeights of one shape and format;
+    route_token: int32 device tensor [R]; expert_offset: E + 1 host integers."""
+    E = len(experts)
+    p0 = experts[0]
+    assert all((p.B, p.G, p.N, p.K) == (p0.B, p0.G, p0.N, p0.K) for p in experts)
+    assert x.dtype in (torch.bfloat16, torch.float16) and x.dim() == 2 and x.shape[1] == p0.K
+    assert route_token.dtype == torch.int32 and route_token.is_cuda
+    off = (C.c_int64 * (E + 1))(*[int(v) for v in expert_offset])
+    ptrs = (C.c_void_p * E)(*[_ptr(p.layout) for p in experts])
+    R = int(expert_offset[-1])
+    assert route_token.numel() == R
+    need = lib().cq_routed_workspace_bytes(p0.B, p0.G, E, off, p0.N, p0.K, mode)
+    if workspace is None:
+        workspace = torch.zeros(max(need, 512), dtype=torch.uint8, device=x.device)
+    y = torch.empty((R, p0.N), dtype=x.dtype, device=x.device)
+    _check(lib().cq_gemm_routed(ptrs, E, p0.B, p0.G, _ptr(x), _ptr(route_token), off, _ptr(y), x.shape[0], p0.N, p0.K, mode,
+                                1 if x.dtype == torch.float16 else 0, _ptr(workspace), workspace.numel(), _stream()),
+           "cq_gemm_routed")
     return y
 
 

@@ -224,6 +224,61 @@ int cq_mlp_swiglu(const void *layout_gate_up, int B_gu, int G_gu, const void *la
     return wrap(e);
 }
 
+// Workspace of the routed product: [gathered rows: R x K model-dtype values][the largest per-matrix cq_gemm workspace].
+static bool routed_offsets_ok(const int64_t *off, int E, int64_t R) {
+    if (!off || off[0] != 0 || off[E] != R) return false;
+    for (int e = 0; e < E; ++e) if (off[e + 1] < off[e]) return false;
+    return true;
+}
+static size_t routed_sub_bytes(const Dims &d, const int64_t *off, int E, int mode) {
+    size_t need = 0;
+    for (int e = 0; e < E; ++e) {
+        const int64_t m = off[e + 1] - off[e];
+        if (m > 0) { const size_t t = plan_workspace(d, m, mode).total; if (t > need) need = t; }
+    }
+    return need;
+}
+
+size_t cq_routed_workspace_bytes(int B, int G, int E, const int64_t *expert_offset_host, int64_t N, int64_t K, int mode) {
+    if (check_format(B, G, N, K) != CQ_OK || E <= 0 || !expert_offset_host || (mode != CQ_MODEL_DTYPE && mode != CQ_DYN_A8)) return 0;
+    const int64_t R = expert_offset_host[E];
+    if (R <= 0 || !routed_offsets_ok(expert_offset_host, E, R)) return 0;
+    return align_up((size_t)R * K * 2, 256) + routed_sub_bytes(make_dims(B, G, N, K), expert_offset_host, E, mode);
+}
+
+int cq_gemm_routed(const void *const *layouts_host, int E, int B, int G, const uint16_t *x, const int32_t *route_token,
+                   const int64_t *expert_offset_host, uint16_t *y_routes, int64_t T, int64_t N, int64_t K, int mode, int act_f16,
+                   void *workspace, size_t workspace_bytes, void *stream) {
+    if (!layouts_host || !x || !route_token || !expert_offset_host || !y_routes || !workspace || E <= 0 || T <= 0)
+        return CQ_ERR_INVALID_ARG;
+    if (mode != CQ_MODEL_DTYPE && mode != CQ_DYN_A8) return CQ_ERR_INVALID_ARG;
+    int st = check_format(B, G, N, K);
+    if (st != CQ_OK) return st;
+    const int64_t R = expert_offset_host[E];
+    if (R <= 0 || !routed_offsets_ok(expert_offset_host, E, R)) return CQ_ERR_INVALID_ARG;
+    for (int e = 0; e < E; ++e) {
+        if (!layouts_host[e]) return CQ_ERR_INVALID_ARG;
+        if (misaligned(layouts_host[e])) return CQ_ERR_ALIGNMENT;
+    }
+    if (misaligned(x) || misaligned(y_routes) || misaligned(workspace) || (K * 2) % 16 != 0 || (N * 2) % 16 != 0) return CQ_ERR_ALIGNMENT;
+    const Dims d = make_dims(B, G, N, K);
+    const size_t xg_bytes = align_up((size_t)R * K * 2, 256), sub = routed_sub_bytes(d, expert_offset_host, E, mode);
+    if (workspace_bytes < xg_bytes + sub) return CQ_ERR_WORKSPACE;
+    st = check_arch();
+    if (st != CQ_OK) return st;
+    uint16_t *xg = reinterpret_cast<uint16_t *>(workspace);
+    cudaError_t e0 = launch_gather_rows(x, route_token, xg, R, T, K, (cudaStream_t)stream);
+    if (e0 != cudaSuccess) return wrap(e0);
+    uint8_t *sub_ws = (uint8_t *)workspace + xg_bytes;
+    for (int e = 0; e < E; ++e) {   // one dispatch per matrix that has routes: its decoded tiles serve all of them
+        const int64_t r0 = expert_offset_host[e], m = expert_offset_host[e + 1] - r0;
+        if (m == 0) continue;
+        st = gemm_any(layouts_host[e], B, G, xg + r0 * K, y_routes + r0 * N, m, N, K, mode, act_f16 != 0, sub_ws, sub, stream);
+        if (st != CQ_OK) return st;
+    }
+    return CQ_OK;
+}
+
 int cq_gemm_status(const void *workspace, size_t workspace_bytes, void *stream) {
     if (!workspace || workspace_bytes < 512) return CQ_ERR_INVALID_ARG;
     // the status word is the first word of every workspace (plan_workspace)

@@ -25,6 +25,9 @@ cudaError_t launch_quantize_a8(const uint16_t *x, int64_t M, int64_t K, int8_t *
 // h[M][2 I] (gate | up, model dtype) -> INT8 carrier of silu(gate) * up in the MMA operand order, and its row scales
 cudaError_t launch_swiglu_quantize_a8(const uint16_t *h, int64_t M, int64_t I, int8_t *x8, int64_t x8_pitch, float *dx,
                                       bool act_f16, cudaStream_t st);
+// routed execution: xg[r] = x[route_token[r]] (zero row for an index outside [0, T))
+cudaError_t launch_gather_rows(const uint16_t *x, const int32_t *route_token, uint16_t *xg, int64_t R, int64_t T, int64_t K,
+                               cudaStream_t st);
 cudaError_t launch_wait_timeout(int *status, long long limit_cycles, cudaStream_t st);
 
 // Workspace carving (all offsets 256-byte aligned).
