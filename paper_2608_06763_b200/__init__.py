@@ -6,7 +6,7 @@ kernels.  There is no CPU fallback: importing works without a GPU (so the build 
 but every compute call needs a CUDA device and the built shared library.
 """
 from .binding import (CQ_DYN_A8, CQ_EFFORT, CQ_FIT_CONTINUOUS, CQ_FIT_JOINT, CQ_MODEL_DTYPE, CubicQuantError, PackedWeights, cq_canonical_code_bytes,
-                      cq_debug_a8_partials, cq_debug_wait_timeout, cq_decode_carriers, cq_decode_levels, cq_decode_weights,
+                      cq_debug_a8_partials, cq_debug_gemm_plan, cq_debug_wait_timeout, cq_decode_carriers, cq_decode_levels, cq_decode_weights,
                       cq_effective_bits, cq_encode, cq_encode_assign, cq_encode_losses, cq_encode_scale, cq_gemm, cq_gemm_host, cq_gemm_routed, cq_gemm_status, cq_gemv_static, cq_layout_bytes, cq_mlp_swiglu, cq_pack_codes, cq_quantize_a8,
                       cq_repack, cq_status_string, cq_unpack, cq_workspace_bytes, cq_workspace_init, lib,
                       library_path)

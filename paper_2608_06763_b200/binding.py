@@ -69,6 +69,8 @@ def lib():
         L.cq_decode_carriers.argtypes = [vp, i, i, i64, i64, vp, vp]
         L.cq_decode_weights.argtypes = [vp, i, i, i64, i64, vp, vp]
         L.cq_debug_a8_partials.argtypes = [vp, i, i, vp, i64, i64, i64, vp, vp]
+        L.cq_debug_gemm_plan.argtypes = [i, i, i64, i64, i64, vp]
+        L.cq_debug_gemm_plan.restype = i
         L.cq_debug_wait_timeout.argtypes = [vp, sz, i64, vp]
         L.cq_debug_wait_timeout.restype = i
         L.cq_encode_assign.argtypes = [vp, i, i, i64, i64, vp, vp, vp, i, vp, vp]
@@ -286,6 +288,13 @@ def cq_debug_a8_partials(pw: PackedWeights, x8: torch.Tensor) -> torch.Tensor:
     _check(lib().cq_debug_a8_partials(_ptr(pw.layout), pw.B, pw.G, _ptr(x8), M, pw.N, pw.K, _ptr(out), _stream()),
            "cq_debug_a8_partials")
     return out
+
+
+def cq_debug_gemm_plan(B: int, G: int, M: int, N: int, K: int) -> dict:
+    """How the model-dtype GEMM (M > 16) spreads a problem over the current device."""
+    out = (C.c_int64 * 4)()
+    _check(lib().cq_debug_gemm_plan(B, G, M, N, K, out), "cq_debug_gemm_plan")
+    return {"token_tile": out[0], "whole_tile_ctas": out[1], "stream_k_ctas": out[2], "stream_k_tiles": out[3]}
 
 
 def cq_debug_wait_timeout(workspace: torch.Tensor, limit_cycles: int = 2_000_000):

@@ -17,7 +17,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libcubicquant.so")
-SOURCES = ["cq_api.cu", "cq_layout.cu", "cq_gemv.cu", "cq_gemm_tc.cu", "cq_gemm_a8_tc.cu", "cq_static.cu", "cq_encode.cu", "cq_routed.cu"]
+SOURCES = ["cq_api.cu", "cq_layout.cu", "cq_gemv.cu", "cq_gemm_tc.cu", "cq_gemm_tc_sk.cu", "cq_gemm_a8_tc.cu", "cq_static.cu", "cq_encode.cu", "cq_routed.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr",
               "-I", INCLUDE, "-I", CSRC]

@@ -24,11 +24,16 @@ Workspace plan_workspace(const Dims &d, int64_t M, int mode) {
     w.status_off = off; off += 256;  // first, so cq_gemm_status finds it without knowing the problem
     // arrival counters: one per 128-row block (small M) or per output tile (split-K GEMM)
     const int64_t bnt = mode == CQ_MODEL_DTYPE ? gemm_tc_token_tile(M) : gemm_a8_token_tile(d, M);
-    const int sk = M <= 16 ? 1 : mode == CQ_MODEL_DTYPE ? gemm_tc_split_k(d, M) : gemm_a8_split_k(d, M);
+    const int sk = M <= 16 || mode == CQ_MODEL_DTYPE ? 1 : gemm_a8_split_k(d, M);
     const size_t n_ctr = (size_t)d.NB * (M > 16 ? (size_t)((M + bnt - 1) / bnt) : 1);
     w.counters_off = off; w.counters_bytes = align_up(n_ctr * 4, 256); off += w.counters_bytes;
     size_t part = (size_t)gp.ctas * 2 * Mc * TILE * 4;   // two partial slots per CTA
     if (sk > 1) { const size_t p2 = (size_t)sk * M * d.NB * TILE * 4; if (p2 > part) part = p2; }
+    if (M > 16 && mode == CQ_MODEL_DTYPE) {   // stream-K: two partial tiles per CTA
+        const TcPlan tp = gemm_tc_plan(d, M);
+        const size_t p2 = tp.stream_k ? (size_t)tp.p2 * 2 * tp.bnt * TILE * 4 : 0;
+        if (p2 > part) part = p2;
+    }
     w.partial_off = off; w.partial_bytes = align_up(part, 256); off += w.partial_bytes;
     if (mode == CQ_DYN_A8) {
         w.x8_off = off; w.x8_bytes = align_up((size_t)(M + 127) / 128 * 128 * Kp, 256); off += w.x8_bytes;
@@ -378,6 +383,16 @@ int cq_decode_weights(const void *layout, int B, int G, int64_t N, int64_t K, fl
     if (!What) return CQ_ERR_INVALID_ARG;
     CQ_DEBUG_PROLOGUE();
     return wrap(launch_decode_weights(layout, d, What, (cudaStream_t)stream));
+}
+
+int cq_debug_gemm_plan(int B, int G, int64_t M, int64_t N, int64_t K, int64_t *plan) {
+    if (!plan || M <= 16) return CQ_ERR_INVALID_ARG;
+    const int st = check_format(B, G, N, K);
+    if (st != CQ_OK) return st;
+    const Dims d = make_dims(B, G, N, K);
+    const TcPlan tp = gemm_tc_plan(d, M);
+    plan[0] = tp.bnt; plan[1] = tp.t_full; plan[2] = tp.p2; plan[3] = (int64_t)d.NB * tp.token_tiles - tp.t_full;
+    return CQ_OK;
 }
 
 int cq_debug_wait_timeout(void *workspace, size_t workspace_bytes, int64_t limit_cycles, void *stream) {

@@ -34,14 +34,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait: false (and a status word) when the barrier did not flip within the limit.
+// `abandon` (optional, shared memory): a flag another thread of the CTA raises when its own wait ran out; this
+// wait then returns false as well, without touching the status word.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *status, int code,
-                                          long long limit = WAIT_LIMIT_CYCLES) {
+                                          long long limit = WAIT_LIMIT_CYCLES, volatile int *abandon = nullptr) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
+        if (abandon && *abandon) return false;
         if (clock64() - t0 > limit) {
             atomicCAS(status, 0, code);
             return false;

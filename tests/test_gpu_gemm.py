@@ -124,6 +124,37 @@ def test_tensor_core_gemm_wide_token_tile(M):
     assert cq.cq_gemm_status(ws) == 0
 
 
+# Stream-K: output tiles shared by several CTAs (partial tiles through the workspace, added in K order by the
+# last CTA to arrive).  (N, K, M): few tiles, each cut into many runs; one tile, ragged in N, K and M; more
+# tiles than SMs, so that whole-tile CTAs and runs share a launch; a 512-token tile with a ragged last tile.
+STREAM_K_SHAPES = [(256, 8192, 40), (100, 4096 + 128, 33), (128 * 150, 4096, 40), (384, 8192, 700)]
+
+
+@pytest.mark.parametrize("act", ["bf16", "f16"])
+@pytest.mark.parametrize("N,K,M", STREAM_K_SHAPES)
+def test_tensor_core_gemm_stream_k(N, K, M, act):
+    B, G = (4, 128) if N != 100 else (3, 64)
+    plan = cq.cq_debug_gemm_plan(B, G, M, N, K)
+    assert plan["stream_k_ctas"] > plan["stream_k_tiles"] > 0, plan   # the shape does share tiles between CTAs
+    if N > 128 * 148:
+        assert plan["whole_tile_ctas"] > 0, plan
+    c = logical_case(N, K, B, G, seed=180 + M)
+    x = datagen.activations(M, K, seed=181, outlier_cols=0.01)      # bf16 bit patterns
+    if act == "f16":
+        x = datagen.bf16_bits_to_f32(x).astype(np.float16).view(np.uint16)
+        xd = torch.from_numpy(x.view(np.float16)).cuda()
+    else:
+        xd = x_to_device(x)
+    ws = torch.zeros(cq.cq_workspace_bytes(B, G, M, N, K, 0), dtype=torch.uint8, device="cuda")
+    y1 = cq.cq_gemm(c.pw, xd, 0, ws).clone()
+    assert cq.cq_gemm_status(ws) == 0
+    y2 = cq.cq_gemm(c.pw, xd, 0, ws).clone()          # the counters were left at zero; fixed order of addition
+    assert torch.equal(y1.view(torch.int16), y2.view(torch.int16))
+    ref = oracle.gemm_model(c.codes, c.s, c.a, c.b, c.B, c.G, c.K, x, act=act)
+    yn = y_to_numpy(y1) if act == "bf16" else y1.cpu().numpy().astype(np.float64)
+    check_y(yn, ref, f"stream-K N={N} K={K} M={M} {act}")
+
+
 @pytest.mark.parametrize("G", [32, 64, 128])
 @pytest.mark.parametrize("B", ALL_B)
 def test_tensor_core_a8_gemm_all_widths_and_groups(B, G):
