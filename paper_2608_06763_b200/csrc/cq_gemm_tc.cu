@@ -31,8 +31,9 @@ int gemm_tc_token_tile(int64_t M) { return M <= 32 ? 32 : M <= 64 ? 64 : M <= 12
 // How the model-dtype GEMM is spread over the SMs.  Whole tiles, one CTA each, fill the SMs round after
 // round.  When the last round would leave many SMs idle, its tiles are cut along K as well (stream-K) and
 // shared by as many CTAs as there are SMs -- if that pays.  In units of one layout tile of main loop: a whole
-// tile costs KT + 4 (pipeline fill, epilogue); a run that shares tiles costs its length + 16 (a second fill, the
-// partial tile's round trip through L2 and, for one CTA per tile, the addition of the partial tiles); and the
+// tile costs KT + 4 (pipeline fill, epilogue); a run that shares tiles costs its length + 16 at the 512-token tile
+// when it crosses from one tile into the next (a second fill, two partial tiles through L2 and, for one CTA per
+// tile, the addition of the partial tiles), + 10 when it does not, less at narrower tiles; and the
 // kernel that can share tiles runs about 5 % slower on every tile than the one that cannot (measured on
 // M = 4096, N = 57344, K = 8192), so the last round has to save more than that.
 TcPlan gemm_tc_plan(const Dims &d, int64_t M) {
@@ -44,10 +45,18 @@ TcPlan gemm_tc_plan(const Dims &d, int64_t M) {
     p.t_full = T; p.p2 = 0;
     if (r != 0) {
         const int64_t V2 = r * d.KT;
-        int64_t p2 = sms;
-        if (p2 > V2 / 4) p2 = V2 / 4;               // at least four layout tiles per run
         const double whole = (double)(d.KT + 4), rounds = (double)(T / sms + 1);
-        if (p2 > r && (whole - ((double)V2 / (double)p2 + 16.0)) / (rounds * whole) > 0.06) { p.t_full = T - r; p.p2 = (int)p2; }
+        // (a) as many runs as SMs: the best balance, but most runs cross from one tile into the next (two fills,
+        //     two partial tiles); (b) every tile cut into the same number of runs: none crosses
+        int64_t pa = sms, pb = r * (sms / r);
+        if (pa > V2 / 4) pa = V2 / 4;               // at least four layout tiles per run
+        if (pb > V2 / 4) pb = r * ((V2 / 4) / r);
+        const double wide = (double)p.bnt / 512.0;   // the partial tiles grow with the token tile
+        const double ca = pa > r ? (double)V2 / (double)pa + 6.0 + 10.0 * wide : 1e30;
+        const double cb = pb > r ? (double)V2 / (double)pb + 4.0 + 6.0 * wide : 1e30;
+        const int64_t p2 = cb <= ca ? pb : pa;
+        const double cost = cb <= ca ? cb : ca;
+        if (p2 > r && (whole - cost) / (rounds * whole) > 0.06) { p.t_full = T - r; p.p2 = (int)p2; }
     }
     p.ctas = (int)(p.t_full + p.p2);
     p.stream_k = p.p2 > 0;
