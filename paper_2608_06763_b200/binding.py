@@ -292,9 +292,10 @@ def cq_debug_a8_partials(pw: PackedWeights, x8: torch.Tensor) -> torch.Tensor:
 
 def cq_debug_gemm_plan(B: int, G: int, M: int, N: int, K: int) -> dict:
     """How the model-dtype GEMM (M > 16) spreads a problem over the current device."""
-    out = (C.c_int64 * 4)()
+    out = (C.c_int64 * 5)()
     _check(lib().cq_debug_gemm_plan(B, G, M, N, K, out), "cq_debug_gemm_plan")
-    return {"token_tile": out[0], "whole_tile_ctas": out[1], "stream_k_ctas": out[2], "stream_k_tiles": out[3]}
+    return {"token_tile": out[0], "whole_tile_ctas": out[1], "stream_k_ctas": out[2], "stream_k_tiles": out[3],
+            "runs_cross_tiles": bool(out[4])}
 
 
 def cq_debug_wait_timeout(workspace: torch.Tensor, limit_cycles: int = 2_000_000):

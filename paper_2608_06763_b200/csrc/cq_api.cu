@@ -29,9 +29,9 @@ Workspace plan_workspace(const Dims &d, int64_t M, int mode) {
     w.counters_off = off; w.counters_bytes = align_up(n_ctr * 4, 256); off += w.counters_bytes;
     size_t part = (size_t)gp.ctas * 2 * Mc * TILE * 4;   // two partial slots per CTA
     if (sk > 1) { const size_t p2 = (size_t)sk * M * d.NB * TILE * 4; if (p2 > part) part = p2; }
-    if (M > 16 && mode == CQ_MODEL_DTYPE) {   // stream-K: two partial tiles per CTA
+    if (M > 16 && mode == CQ_MODEL_DTYPE) {   // stream-K: two partial tiles per run
         const TcPlan tp = gemm_tc_plan(d, M);
-        const size_t p2 = tp.stream_k ? (size_t)tp.p2 * 2 * tp.bnt * TILE * 4 : 0;
+        const size_t p2 = (size_t)tp.p2 * 2 * tp.bnt * TILE * 4;
         if (p2 > part) part = p2;
     }
     w.partial_off = off; w.partial_bytes = align_up(part, 256); off += w.partial_bytes;
@@ -392,6 +392,7 @@ int cq_debug_gemm_plan(int B, int G, int64_t M, int64_t N, int64_t K, int64_t *p
     const Dims d = make_dims(B, G, N, K);
     const TcPlan tp = gemm_tc_plan(d, M);
     plan[0] = tp.bnt; plan[1] = tp.t_full; plan[2] = tp.p2; plan[3] = (int64_t)d.NB * tp.token_tiles - tp.t_full;
+    plan[4] = tp.crossing;
     return CQ_OK;
 }
 

@@ -29,34 +29,41 @@ int gemm_tc_available() { return 1; }
 // Token tile of the model-dtype GEMM for M rows.
 int gemm_tc_token_tile(int64_t M) { return M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : M <= 256 ? 256 : 512; }
 // How the model-dtype GEMM is spread over the SMs.  Whole tiles, one CTA each, fill the SMs round after
-// round.  When the last round would leave many SMs idle, its tiles are cut along K as well (stream-K) and
-// shared by as many CTAs as there are SMs -- if that pays.  In units of one layout tile of main loop: a whole
-// tile costs KT + 4 (pipeline fill, epilogue); a run that shares tiles costs its length + 16 at the 512-token tile
-// when it crosses from one tile into the next (a second fill, two partial tiles through L2 and, for one CTA per
-// tile, the addition of the partial tiles), + 10 when it does not, less at narrower tiles; and the
-// kernel that can share tiles runs about 5 % slower on every tile than the one that cannot (measured on
-// M = 4096, N = 57344, K = 8192), so the last round has to save more than that.
+// round.  When the last round would leave SMs idle, its r tiles are cut along K as well (stream-K) -- if that
+// pays.  In units of one layout tile of main loop: a whole tile costs KT + 4 (pipeline fill, epilogue).
+//   (b) every tile cut into the same number s of runs, so that a run lies inside its tile: a run costs its
+//       length + 4 .. 10 (the fill, the partial tile's trip through L2 and, for one CTA per tile, the addition
+//       of the partial tiles; the more the wider the token tile), and r s runs take ceil(r s / SMs) rounds;
+//   (a) one run per SM, cut anywhere: the best balance, but most runs cross from one tile into the next (two
+//       fills, two partial tiles: length + 6 .. 16).
+// The kernel that can share tiles runs about 5 % slower on every tile of the launch than the one that cannot
+// (measured at M = 4096, N = 57344, K = 8192, and at M = 1024, N = 6144, K = 4096; merely compiling the partial-tile
+// code into the kernel costs that much), so it is a separate instantiation and sharing has to save more.
 TcPlan gemm_tc_plan(const Dims &d, int64_t M) {
     TcPlan p;
     p.bnt = gemm_tc_token_tile(M);
     p.token_tiles = (int)((M + p.bnt - 1) / p.bnt);
     const int64_t T = (int64_t)d.NB * p.token_tiles, sms = sm_count();
     const int64_t r = T % sms;                      // tiles of the last, partial round
-    p.t_full = T; p.p2 = 0;
+    p.t_full = T; p.p2 = 0; p.crossing = 0;
     if (r != 0) {
         const int64_t V2 = r * d.KT;
-        const double whole = (double)(d.KT + 4), rounds = (double)(T / sms + 1);
-        // (a) as many runs as SMs: the best balance, but most runs cross from one tile into the next (two fills,
-        //     two partial tiles); (b) every tile cut into the same number of runs: none crosses
-        int64_t pa = sms, pb = r * (sms / r);
-        if (pa > V2 / 4) pa = V2 / 4;               // at least four layout tiles per run
-        if (pb > V2 / 4) pb = r * ((V2 / 4) / r);
         const double wide = (double)p.bnt / 512.0;   // the partial tiles grow with the token tile
-        const double ca = pa > r ? (double)V2 / (double)pa + 6.0 + 10.0 * wide : 1e30;
-        const double cb = pb > r ? (double)V2 / (double)pb + 4.0 + 6.0 * wide : 1e30;
-        const int64_t p2 = cb <= ca ? pb : pa;
-        const double cost = cb <= ca ? cb : ca;
-        if (p2 > r && (whole - cost) / (rounds * whole) > 0.06) { p.t_full = T - r; p.p2 = (int)p2; }
+        const double whole = (double)(d.KT + 4), all = (double)(T / sms + 1) * whole;
+        double best = 1e30;
+        int64_t best_p2 = 0;
+        int best_crossing = 0;
+        for (int64_t s = 2; s <= 16 && s * 4 <= d.KT; ++s) {
+            const double c = (double)((r * s + sms - 1) / sms) * ((double)d.KT / (double)s + 4.0 + 6.0 * wide);
+            if (c < best) { best = c; best_p2 = r * s; best_crossing = 0; }
+        }
+        int64_t pa = sms;
+        if (pa > V2 / 4) pa = V2 / 4;               // at least four layout tiles per run
+        if (pa > r) {
+            const double c = (double)V2 / (double)pa + 6.0 + 10.0 * wide;
+            if (c < best) { best = c; best_p2 = pa; best_crossing = 1; }
+        }
+        if (best_p2 > 0 && (whole - best) / all > 0.06) { p.p2 = (int)best_p2; p.crossing = best_crossing; p.t_full = T - r; }
     }
     p.ctas = (int)(p.t_full + p.p2);
     p.stream_k = p.p2 > 0;

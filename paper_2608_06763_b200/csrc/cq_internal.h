@@ -72,7 +72,7 @@ GemvPlan gemv_plan(const Dims &d, int64_t M, int mode);
 cudaError_t launch_gemv(const void *layout, const Dims &d, const uint16_t *x, uint16_t *y, int64_t M, int mode,
                         bool act_f16, uint8_t *ws, const Workspace &plan, cudaStream_t st, bool prequantized = false);
 int gemm_tc_token_tile(int64_t M);
-struct TcPlan { int bnt, token_tiles, ctas, stream_k, p2; int64_t t_full; };
+struct TcPlan { int bnt, token_tiles, ctas, stream_k, p2, crossing; int64_t t_full; };
 TcPlan gemm_tc_plan(const Dims &d, int64_t M);
 int gemm_a8_token_tile(const Dims &d, int64_t M);
 int gemm_a8_split_k(const Dims &d, int64_t M);

@@ -67,7 +67,7 @@ def test_argument_errors_are_found_before_any_launch():
 def test_gemm_plan_shares_the_last_round_only_when_it_pays():
     """Host logic of the model-dtype GEMM's schedule (148 SMs are assumed when no device can be asked)."""
     L = cq.lib()
-    plan = (ctypes.c_int64 * 4)()
+    plan = (ctypes.c_int64 * 5)()
 
     def ask(B, G, M, N, K):
         assert L.cq_debug_gemm_plan(B, G, M, N, K, plan) == 0
@@ -76,16 +76,17 @@ def test_gemm_plan_shares_the_last_round_only_when_it_pays():
     assert L.cq_debug_gemm_plan(4, 128, 16, 4096, 4096, plan) == -1       # M <= 16 is the small-M kernel's
     assert L.cq_debug_gemm_plan(4, 128, 64, 4096, 4096, None) == -1
     for (M, N, K) in [(1024, 28672, 4096), (1024, 4096, 14336), (4096, 8192, 28672), (40, 256, 8192), (33, 100, 4224),
-                      (4096, 57344, 8192), (1024, 6144, 4096), (17, 128, 128), (300, 200, 1024)]:
-        bnt, whole, runs, shared = ask(4, 128, M, N, K)
+                      (4096, 57344, 8192), (1024, 6144, 4096), (17, 128, 128), (300, 200, 1024), (32, 28672, 4096)]:
+        bnt, whole, runs, shared, crossing = ask(4, 128, M, N, K)
         tiles = -(-N // 128) * -(-M // bnt)
         kt = -(-K // 128)
         assert bnt in (32, 64, 128, 256, 512) and whole + shared == tiles
         if runs:
-            assert shared < runs <= 148 and whole % 148 == 0     # whole rounds, then one round of runs
+            assert shared < runs and whole % 148 == 0            # whole rounds, then the runs
             assert shared * kt >= 4 * runs                       # at least four layout tiles per run
+            assert runs <= 148 if crossing else runs % shared == 0   # one run per SM, or the same number per tile
         else:
-            assert shared == 0
-    assert ask(4, 128, 1024, 28672, 4096) == [512, 444, 32, 4]        # three whole rounds, four tiles shared by 32 CTAs
+            assert shared == 0 and not crossing
+    assert ask(4, 128, 1024, 28672, 4096) == [512, 444, 32, 4, 0]     # three whole rounds, four tiles cut into eight runs each
     assert ask(4, 128, 4096, 57344, 8192)[2] == 0                     # 24 rounds and a bit: sharing would not pay
     assert ask(4, 128, 17, 128, 128)[2] == 0                          # one layout tile of K cannot be cut

@@ -125,17 +125,22 @@ def test_tensor_core_gemm_wide_token_tile(M):
 
 
 # Stream-K: output tiles shared by several CTAs (partial tiles through the workspace, added in K order by the
-# last CTA to arrive).  (N, K, M): few tiles, each cut into many runs; one tile, ragged in N, K and M; more
-# tiles than SMs, so that whole-tile CTAs and runs share a launch; a 512-token tile with a ragged last tile.
-STREAM_K_SHAPES = [(256, 8192, 40), (100, 4096 + 128, 33), (128 * 150, 4096, 40), (384, 8192, 700)]
+# last CTA to arrive).  (N, K, M, runs cross tiles): few tiles, each cut into many runs; one tile, ragged in N, K
+# and M; more tiles than SMs, so that whole-tile CTAs and runs share a launch; a 512-token tile with a ragged last
+# tile; a last round of 76 tiles shared by one run per SM, so that runs cross from one tile into the next (the
+# kernel of cq_gemm_tc_sk.cu).
+STREAM_K_SHAPES = [(256, 8192, 40, False), (100, 4096 + 128, 33, False), (128 * 150, 4096, 40, False),
+                   (384, 8192, 700, False), (128 * (148 + 76), 2048, 20, True)]
 
 
 @pytest.mark.parametrize("act", ["bf16", "f16"])
-@pytest.mark.parametrize("N,K,M", STREAM_K_SHAPES)
-def test_tensor_core_gemm_stream_k(N, K, M, act):
+@pytest.mark.parametrize("N,K,M,crossing", STREAM_K_SHAPES)
+def test_tensor_core_gemm_stream_k(N, K, M, crossing, act):
     B, G = (4, 128) if N != 100 else (3, 64)
     plan = cq.cq_debug_gemm_plan(B, G, M, N, K)
     assert plan["stream_k_ctas"] > plan["stream_k_tiles"] > 0, plan   # the shape does share tiles between CTAs
+    if torch.cuda.get_device_properties(0).multi_processor_count == 148:
+        assert plan["runs_cross_tiles"] == crossing, plan
     if N > 128 * 148:
         assert plan["whole_tile_ctas"] > 0, plan
     c = logical_case(N, K, B, G, seed=180 + M)
