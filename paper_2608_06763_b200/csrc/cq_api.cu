@@ -24,11 +24,14 @@ Workspace plan_workspace(const Dims &d, int64_t M, int mode) {
     w.status_off = off; off += 256;  // first, so cq_gemm_status finds it without knowing the problem
     // arrival counters: one per 128-row block (small M) or per output tile (split-K GEMM)
     const int64_t bnt = mode == CQ_MODEL_DTYPE ? gemm_tc_token_tile(M) : gemm_a8_token_tile(d, M);
-    const int sk = M <= 16 || mode == CQ_MODEL_DTYPE ? 1 : gemm_a8_split_k(d, M);
     const size_t n_ctr = (size_t)d.NB * (M > 16 ? (size_t)((M + bnt - 1) / bnt) : 1);
     w.counters_off = off; w.counters_bytes = align_up(n_ctr * 4, 256); off += w.counters_bytes;
     size_t part = (size_t)gp.ctas * 2 * Mc * TILE * 4;   // two partial slots per CTA
-    if (sk > 1) { const size_t p2 = (size_t)sk * M * d.NB * TILE * 4; if (p2 > part) part = p2; }
+    if (M > 16 && mode == CQ_DYN_A8) {        // tiles of the last round cut into slices: one partial tile per slice
+        const A8Plan ap = gemm_a8_plan(d, M);
+        const size_t p2 = ap.slices > 1 ? (size_t)((int64_t)d.NB * ap.token_tiles - ap.t_full) * ap.slices * ap.bn * TILE * 4 : 0;
+        if (p2 > part) part = p2;
+    }
     if (M > 16 && mode == CQ_MODEL_DTYPE) {   // stream-K: two partial tiles per run
         const TcPlan tp = gemm_tc_plan(d, M);
         const size_t p2 = (size_t)tp.p2 * 2 * tp.bnt * TILE * 4;

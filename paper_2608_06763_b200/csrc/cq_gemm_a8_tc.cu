@@ -22,20 +22,37 @@
 namespace cq {
 
 // Token tile of the Dynamic-A8 GEMM (two accumulator buffers of (128 / G) x tile columns fill at most
-// the 512 TMEM columns), and its split-K factor for grids that would leave most SMs idle.
+// the 512 TMEM columns).
 int gemm_a8_token_tile(const Dims &d, int64_t M) {
     const int bmax = 256 / d.gpt;
     const int bn = M <= 64 ? 64 : M <= 128 ? 128 : 256;
     return bn < bmax ? bn : bmax;
 }
-int gemm_a8_split_k(const Dims &d, int64_t M) {
-    const int64_t bnt = gemm_a8_token_tile(d, M);
-    const int64_t ctas = (int64_t)d.NB * ((M + bnt - 1) / bnt);
-    if (ctas >= 100 || M > 256) return 1;
-    int64_t sk = sm_count() / ctas;
-    if (sk > 8) sk = 8;
-    if (sk > d.KT / 4) sk = d.KT / 4;   // at least four layout tiles per slice
-    return sk < 1 ? 1 : (int)sk;
+// How the Dynamic-A8 GEMM is spread over the SMs: whole tiles, one CTA each, round after round; when the last
+// round would leave SMs idle, each of its r tiles is cut along K into the same number s of slices (one CTA each;
+// the last CTA of a tile to arrive adds the partial tiles in K order).  In units of one 128-wide K block of main
+// loop: a whole tile costs KT + 3, a slice KT / s + 3 + up to 4 for the partial tile's trip through L2 and its share
+// of the addition; r s slices take ceil(r s / SMs) rounds.  Slices are used when that saves more than 3 % of the
+// whole launch.
+A8Plan gemm_a8_plan(const Dims &d, int64_t M) {
+    A8Plan p;
+    p.bn = gemm_a8_token_tile(d, M);
+    p.token_tiles = (int)((M + p.bn - 1) / p.bn);
+    const int64_t T = (int64_t)d.NB * p.token_tiles, sms = sm_count();
+    const int64_t r = T % sms;
+    p.t_full = T; p.slices = 1;
+    if (r != 0) {
+        const double wide = (double)p.bn / 256.0;
+        const double whole = (double)(d.KT + 3), all = (double)(T / sms + 1) * whole;
+        double best = whole;
+        for (int64_t s = 2; s <= 8 && s * 4 <= d.KT; ++s) {
+            const double c = (double)((r * s + sms - 1) / sms) * ((double)d.KT / (double)s + 3.0 + 4.0 * wide);
+            if (c < best) { best = c; p.slices = (int)s; }
+        }
+        if ((whole - best) / all > 0.03) p.t_full = T - r; else p.slices = 1;
+    }
+    p.ctas = (int)(p.t_full + (T - p.t_full) * p.slices);
+    return p;
 }
 
 namespace {
@@ -57,8 +74,10 @@ struct A8Params {
     Dims d;
     int M;
     int raw_stage_bytes;
-    float *partial;       // split-K: fp32 partial sums [SK][M][Np] (before the d_x / 127 factor)
-    int *counters;        // split-K: arrival counters, one per (row block, token tile)
+    float *partial;       // sliced tiles: fp32 partial tiles [shared tile][slice][BN][128] (before the d_x / 127 factor)
+    int *counters;        // sliced tiles: arrival counters, one per output tile
+    int t_full;           // CTAs 0 .. t_full - 1 compute one whole tile each (tile = mt * NB + nb)
+    int slices;           // every later tile is cut along K into this many slices, one CTA each
     bool f16;             // y is written as binary16 instead of bfloat16
 };
 
@@ -93,10 +112,22 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
 
     const Dims &d = prm.d;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int nb = blockIdx.x, mt = blockIdx.y;
-    // split-K: blockIdx.z takes the layout tiles [kt0, kt0 + KT) of the K range
-    const int kt0 = (int)(((int64_t)d.KT * blockIdx.z) / gridDim.z);
-    const int KT = (int)(((int64_t)d.KT * (blockIdx.z + 1)) / gridDim.z) - kt0;
+    // This CTA's tile and, for a tile of the last round, its slice z of nz: the layout tiles [kt0, kt0 + KT)
+    int kt0, KT, p_nb, p_mt;
+    {
+        const int bid = (int)blockIdx.x;
+        const int nz = bid < prm.t_full ? 1 : prm.slices;
+        const int tile_id = bid < prm.t_full ? bid : prm.t_full + (bid - prm.t_full) / prm.slices;
+        const int z = bid < prm.t_full ? 0 : (bid - prm.t_full) % prm.slices;
+        p_mt = tile_id / d.NB; p_nb = tile_id - p_mt * d.NB;
+        kt0 = (int)(((int64_t)d.KT * z) / nz);
+        KT = (int)(((int64_t)d.KT * (z + 1)) / nz) - kt0;
+        if (threadIdx.x == 0) {   // what only the epilogue needs is parked in shared memory (set up below, before the barrier)
+            uint32_t *park = reinterpret_cast<uint32_t *>(acc_empty + 2);
+            park[4] = (uint32_t)nz; park[5] = (uint32_t)z; park[6] = (uint32_t)tile_id; park[7] = (uint32_t)p_nb; park[8] = (uint32_t)p_mt;
+        }
+    }
+    const int nb = p_nb, mt = p_mt;   // the producer's coordinates
 
     if ((smem_u32(smem) & 1023u) != 0) {
         if (threadIdx.x == 0) atomicCAS(prm.status, 0, 9);
@@ -109,6 +140,7 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
         fence_barrier_init();
         tmem_slot[2] = 0;   // the work warps' "a wait gave up" flag
         tmem_slot[3] = prm.f16 ? 1u : 0u;   // the output dtype, parked in shared memory: a register held across the main loop is one too many
+        // tmem_slot[4 .. 8]: slice count, slice, tile, row block and token tile of this CTA (written above)
     }
     if (threadIdx.x < 128) sT[threadIdx.x] = __fdiv_rn((float)threadIdx.x, (float)Mx);  // the pinned t = i / M
     if (warp == 1) {
@@ -293,21 +325,28 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
             }
         }
         if (!*gave_up) {
-            const int64_t n = (int64_t)nb * TILE + drow;
-            if (n < d.N || gridDim.z > 1) {   // partial sums of padding channels are written too (zeros), never read back as y
+            const int e_nb = (int)*reinterpret_cast<volatile uint32_t *>(tmem_slot + 7);
+            const int e_mt = (int)*reinterpret_cast<volatile uint32_t *>(tmem_slot + 8);
+            const int64_t n = (int64_t)e_nb * TILE + drow;
+            const int e_nz = (int)*reinterpret_cast<volatile uint32_t *>(tmem_slot + 4);
+            if (n < d.N || e_nz > 1) {   // partial sums of padding channels are written too (zeros), never read back as y
                 // the output dtype is decided once, outside the loop over the 64 accumulators (a select inside it
                 // costs the registers this kernel does not have)
+                // partial tile of this slice: [token of the tile][128 channels]
+                const int e_z = (int)*reinterpret_cast<volatile uint32_t *>(tmem_slot + 5);
+                const int e_tile = (int)*reinterpret_cast<volatile uint32_t *>(tmem_slot + 6);
+                float *pslot = prm.partial + ((size_t)(e_tile - prm.t_full) * prm.slices + e_z) * (size_t)(BN * TILE) + drow;
                 auto store_all = [&](auto f16c) {
                     constexpr bool F16 = decltype(f16c)::value;
 #pragma unroll
                     for (int i = 0; i < QCOLS; ++i) {
-                        const int64_t m = (int64_t)mt * BN + cq4 * QCOLS + i;
+                        const int64_t m = (int64_t)e_mt * BN + cq4 * QCOLS + i;
                         if (m < prm.M) {
-                            if (gridDim.z == 1) {
+                            if (e_nz == 1) {
                                 const float v = acc[i] * (prm.dx[m] * (1.0f / 127.0f));
                                 prm.y[m * d.N + n] = float_to_act(v, F16);
                             } else {
-                                prm.partial[((size_t)blockIdx.z * prm.M + m) * ((size_t)d.NB * TILE) + n] = acc[i];
+                                pslot[(size_t)(cq4 * QCOLS + i) * TILE] = acc[i];
                             }
                         }
                     }
@@ -323,29 +362,31 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
-    if (gridDim.z > 1) {
-        // split-K combine: the last CTA of this output tile to arrive adds the slices in slice order and
-        // applies d_x / 127.  The barrier above ordered the CTA's partial stores before thread 0's release.
+    if (*reinterpret_cast<volatile uint32_t *>(tmem_slot + 4) > 1) {
+        // The last CTA of this output tile to arrive adds the slices in K order and applies d_x / 127.  The barrier
+        // above ordered the CTA's partial stores before thread 0's release.  (Tile, slice count and position are read
+        // back from shared memory: held in registers they would stay live across the main loop.)
+        const int nz = (int)*reinterpret_cast<volatile uint32_t *>(tmem_slot + 4), tile_id = (int)*reinterpret_cast<volatile uint32_t *>(tmem_slot + 6);
+        const int nb = (int)*reinterpret_cast<volatile uint32_t *>(tmem_slot + 7), mt = (int)*reinterpret_cast<volatile uint32_t *>(tmem_slot + 8);
         volatile int *s_last_p = reinterpret_cast<volatile int *>(tmem_slot + 1);   // scratch word after the TMEM slot
-        int *ctr = prm.counters + (nb * gridDim.y + mt);
+        int *ctr = prm.counters + tile_id;
         if (threadIdx.x == 0) {
             int old;
             asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(ctr) : "memory");
-            *s_last_p = (old == (int)gridDim.z - 1);
+            *s_last_p = (old == nz - 1);
         }
         __syncthreads();
         if (*s_last_p) {
-            const size_t Np = (size_t)d.NB * TILE;
             const bool out_f16 = *reinterpret_cast<volatile uint32_t *>(tmem_slot + 3) != 0;
             constexpr int QUADS = BN * TILE / 4;   // four consecutive channels of one token per 128-bit load
+            const float4 *src = reinterpret_cast<const float4 *>(prm.partial + (size_t)(tile_id - prm.t_full) * prm.slices * (size_t)(BN * TILE));
             for (int qd = threadIdx.x; qd < QUADS; qd += A8_THREADS) {
                 const int64_t m = (int64_t)mt * BN + qd / (TILE / 4), n = (int64_t)nb * TILE + (qd % (TILE / 4)) * 4;
                 if (m >= prm.M) continue;
                 float4 v[8];
 #pragma unroll
                 for (int q = 0; q < 8; ++q)
-                    v[q] = q < (int)gridDim.z ? __ldcg(reinterpret_cast<const float4 *>(prm.partial + ((size_t)q * prm.M + m) * Np + n))
-                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+                    v[q] = q < nz ? __ldcg(src + (size_t)q * QUADS + qd) : make_float4(0.f, 0.f, 0.f, 0.f);
                 float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                 for (int q = 0; q < 8; ++q) { sum.x += v[q].x; sum.y += v[q].y; sum.z += v[q].z; sum.w += v[q].w; }  // slice order
@@ -385,8 +426,10 @@ cudaError_t launch_a8(const void *layout, const Dims &d, const int8_t *x8, int64
     static std::atomic<uint64_t> attr_done{0};   // per kernel instantiation: the devices it has been set on
     cudaError_t ea = ensure_func_attr(kern, attr_done, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (ea != cudaSuccess) return ea;
-    dim3 grid((unsigned)d.NB, (unsigned)((M + BN - 1) / BN), (unsigned)gemm_a8_split_k(d, M));
-    kern<<<grid, A8_THREADS, smem, st>>>(xmap, p);
+    const A8Plan plan = gemm_a8_plan(d, M);
+    if (plan.bn != BN) return cudaErrorInvalidConfiguration;
+    p.t_full = (int)plan.t_full; p.slices = plan.slices;
+    kern<<<dim3((unsigned)plan.ctas), A8_THREADS, smem, st>>>(xmap, p);
     return cudaGetLastError();
 }
 

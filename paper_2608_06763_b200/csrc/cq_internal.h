@@ -33,7 +33,7 @@ cudaError_t launch_wait_timeout(int *status, long long limit_cycles, cudaStream_
 // Workspace carving (all offsets 256-byte aligned).
 struct Workspace {
     size_t counters_off, counters_bytes;   // int32 arrival counters, one per 128-row block
-    size_t partial_off, partial_bytes;     // fp32 split-K partial sums: small M [CTA][2][M][128]; model-dtype GEMM [CTA][2][BNT][128]; A8 GEMM [slice][M][Np]
+    size_t partial_off, partial_bytes;     // fp32 split-K partial sums: small M [CTA][2][M][128]; model-dtype GEMM [CTA][2][BNT][128]; A8 GEMM [shared tile][slice][BN][128]
     size_t x8_off, x8_bytes;               // Dynamic A8: int8 activation carrier [M][Kp]
     size_t dx_off, dx_bytes;               // Dynamic A8: row scales [M]
     size_t status_off;                     // int32 device status word (bounded waits report here)
@@ -75,7 +75,8 @@ int gemm_tc_token_tile(int64_t M);
 struct TcPlan { int bnt, token_tiles, ctas, stream_k, p2, crossing; int64_t t_full; };
 TcPlan gemm_tc_plan(const Dims &d, int64_t M);
 int gemm_a8_token_tile(const Dims &d, int64_t M);
-int gemm_a8_split_k(const Dims &d, int64_t M);
+struct A8Plan { int bn, token_tiles, slices, ctas; int64_t t_full; };
+A8Plan gemm_a8_plan(const Dims &d, int64_t M);
 
 // offline encoder steps (cq_encode.cu)
 cudaError_t launch_encode_assign(const float *W, int B, int G, int64_t N, int64_t K, const float *scale, const uint16_t *a,
