@@ -282,6 +282,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                 w3_lo = w3_table(*(const uint2 *)prow, prm.f16);
                 w3_hi = w3_table(*(const uint2 *)(prow + 8 * GPT * 8), prm.f16);
             }
+            // G = 128: one group spans the tile, so its coefficients are formed once per tile, not once per 64-wide block
+            RowCoef tc_lo{}, tc_hi{};
+            bool tfix = false;
+            if constexpr (B != 3 && G == 128) {
+                const uint2 q_lo = *(const uint2 *)prow, q_hi = *(const uint2 *)(prow + 8 * GPT * 8);
+                tc_lo = make_coef<B>(q_lo); tc_hi = make_coef<B>(q_hi);
+                tfix = B > 1 && __any_sync(0xffffffffu, (q_lo.x | q_hi.x) >> 31);
+            }
 #pragma unroll 1
             for (int half_k = 0; half_k < 2; ++half_k) {
                 const int kb = kbc++, s = kb % STAGES;
@@ -308,8 +316,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                         });
                         return;
                     }
-                    const RowCoef c_lo = make_coef<B>(p_lo), c_hi = make_coef<B>(p_hi);
-                    const bool fix = B > 1 && __any_sync(0xffffffffu, (p_lo.x | p_hi.x) >> 31);  // reserved pattern present
+                    RowCoef c_lo, c_hi;
+                    bool fix;   // reserved pattern present
+                    if constexpr (G == 128) { c_lo = tc_lo; c_hi = tc_hi; fix = tfix; }
+                    else { c_lo = make_coef<B>(p_lo); c_hi = make_coef<B>(p_hi); fix = B > 1 && __any_sync(0xffffffffu, (p_lo.x | p_hi.x) >> 31); }
                     auto emit = [&](auto fx, auto hx) {
                         constexpr bool FIX = decltype(fx)::value, F16 = decltype(hx)::value;
                         static_for<2>([&](auto jc) {
