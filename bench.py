@@ -358,6 +358,19 @@ def extra_suites(torch, cq, datagen, stream, peaks):
         if c["model_over_a8"] > 1.0 and key not in first:
             first[key] = c["M"]
     out["crossover_first_M_where_a8_is_faster"] = first
+    # ---- the mid-M target: both GEMMs at M = 1024 on the four shapes (W4 G128), as fractions of the measured peaks
+    shape_of = {name: (K, N) for name, K, N in datagen.LLAMA8B_SHAPES}
+    mid = []
+    for c in cross:
+        if c["M"] == 1024 and c["B"] == 4:
+            K, N = shape_of[c["shape"]]
+            tf, to = 2.0 * 1024 * N * K / (c["us_model"] * 1e-6) / 1e12, 2.0 * 1024 * N * K / (c["us_a8"] * 1e-6) / 1e12
+            mid.append({"shape": c["shape"], "K": K, "N": N, "M": 1024, "tflops_model": round(tf, 1),
+                        "frac_of_measured_bf16_burst": round(tf / peaks["bf16_tflops"], 4), "tops_a8": round(to, 1),
+                        "frac_of_measured_int8": round(to / i8["tops"], 4)})
+    out["gemm_m1024_w4g128"] = {"rows": mid, "target_frac": TARGET_GEMM_FRAC,
+                                "target_met_model_dtype": all(r["frac_of_measured_bf16_burst"] >= TARGET_GEMM_FRAC for r in mid),
+                                "target_met_a8": all(r["frac_of_measured_int8"] >= TARGET_GEMM_FRAC for r in mid)}
     # ---- compact summaries of the two tensor-core kernels (W4 G128 gate_up 8192 -> 57344, M = 4096)
     gm = next(r for r in gemm if r["shape"] == "gate_up" and r["B"] == 4 and r["mode"] == "model_dtype")
     ga = next(r for r in gemm if r["shape"] == "gate_up" and r["B"] == 4 and r["mode"] == "dyn_a8")
