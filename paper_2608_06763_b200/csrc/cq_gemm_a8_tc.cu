@@ -1,8 +1,10 @@
 // Large-M Dynamic-A8 GEMM on tcgen05 (Section 5.4): INT8 activation carriers x INT8 weight
 // carriers -> int32 group partials in TMEM -> fp32 rescale by s_g (and d_x / 127 at the end).
 //
-// CTA = 128 output channels x BN tokens, K (or one split-K slice of it) walked in 128-wide blocks (one layout tile).
-//   warp 0       producer: bulk copy of the raw layout tile, TMA of the x8 tile [BN x 128] (swizzled)
+// CTA = 128 output channels x BN tokens, K (or one slice of it, for a tile of the last round) walked in 128-wide
+// blocks (one layout tile).
+//   warp 0       TMA of the x8 tiles [BN x 128] (swizzled) into a ring of two stages
+//   warp 18      bulk copies of the raw layout tiles into their own ring (2-4 deep)
 //   warp 1       TMEM allocation, tcgen05.mma kind::i8 (K = 32 per instruction); every group of
 //                the block accumulates into its own BN columns of one of two TMEM buffers
 //   warps 2..17  work warps, two jobs per K block, interleaved so the tensor core never waits on both:
@@ -60,9 +62,17 @@ namespace {
 using namespace tc;
 
 constexpr int A8_WORK_WARPS = 16;
-constexpr int A8_THREADS = 32 * (2 + A8_WORK_WARPS);
+constexpr int A8_THREADS = 32 * (3 + A8_WORK_WARPS);   // producer of activations, MMA issuer, work warps, producer of raw tiles
 constexpr int A8_STAGES = 2;     // operand stages (one 128-wide k block each)
-constexpr int A8_RAW_STAGES = 2;
+// Raw layout tiles in flight per CTA: as many as the shared memory left by the rest holds, two to four.
+constexpr int a8_raw_stage_bytes(int B, int G) { return (2048 * B + 1024 * (TILE / G) + 1023) / 1024 * 1024; }
+constexpr int a8_fixed_smem(int B, int G, int BN) {
+    return 2 * (128 * 128 + BN * 128) + 8 * 2 * 16 * carrier_table_stride(B) + 8 * 128 * (TILE / G) * 4 + 512 + 256;
+}
+constexpr int a8_raw_stages(int B, int G, int BN) {
+    const int n = (226 * 1024 - a8_fixed_smem(B, G, BN)) / a8_raw_stage_bytes(B, G);
+    return n > 4 ? 4 : n < 2 ? 2 : n;
+}
 constexpr int A8_SRING = 8;      // ring of per-block scale snapshots for the drain warps
 constexpr int A8_A_STAGE_BYTES = 128 * 128;
 
@@ -96,6 +106,7 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
     constexpr uint32_t ACC_COLS = GPT * BN;       // columns of one accumulator buffer
     constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;  // 512
     constexpr int QCOLS = BN / 4;                 // columns per work thread in the drain
+    constexpr int A8_RAW_STAGES = a8_raw_stages(B, G, BN);
     static_assert(TMEM_COLS <= 512 && (TMEM_COLS & (TMEM_COLS - 1)) == 0, "TMEM columns");
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t *sA = smem;
@@ -153,20 +164,29 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ===== producer
+        // ===== producer of the activation tiles: only the wait for the stage stands between the MMAs that free it
+        // and the TMA that refills it (with two stages that latency is on the critical path)
         if (lane == 0) {
-            const uint8_t *tiles = prm.layout + ((size_t)nb * d.KT + kt0) * (size_t)d.tile_bytes;
             bool ok = true;
             for (int t = 0; t < KT && ok; ++t) {
-                const int rs = t % A8_RAW_STAGES, s = t % A8_STAGES;
-                if (t >= A8_RAW_STAGES) ok = mbar_wait(&raw_empty[rs], ((t / A8_RAW_STAGES) - 1) & 1, prm.status, 11);
-                if (!ok) break;
-                mbar_arrive_expect_tx(&raw_full[rs], (uint32_t)d.tile_bytes);
-                bulk_load(sRaw + rs * prm.raw_stage_bytes, tiles + (size_t)t * d.tile_bytes, (uint32_t)d.tile_bytes, &raw_full[rs]);
+                const int s = t % A8_STAGES;
                 if (t >= A8_STAGES) ok = mbar_wait(&st_empty[s], ((t / A8_STAGES) - 1) & 1, prm.status, 12);
                 if (!ok) break;
                 mbar_arrive_expect_tx(&b_full[s], B_STAGE_BYTES);
                 tma_load_2d(sB + s * B_STAGE_BYTES, &xmap, &b_full[s], (kt0 + t) * 128, mt * BN);
+            }
+        }
+    } else if (warp == 2 + A8_WORK_WARPS) {
+        // ===== producer of the raw layout tiles (its own warp: a wait for the work warps never delays an activation tile)
+        if (lane == 0) {
+            const uint8_t *tiles = prm.layout + ((size_t)nb * d.KT + kt0) * (size_t)d.tile_bytes;
+            bool ok = true;
+            for (int t = 0; t < KT && ok; ++t) {
+                const int rs = t % A8_RAW_STAGES;
+                if (t >= A8_RAW_STAGES) ok = mbar_wait(&raw_empty[rs], ((t / A8_RAW_STAGES) - 1) & 1, prm.status, 11);
+                if (!ok) break;
+                mbar_arrive_expect_tx(&raw_full[rs], (uint32_t)d.tile_bytes);
+                bulk_load(sRaw + rs * prm.raw_stage_bytes, tiles + (size_t)t * d.tile_bytes, (uint32_t)d.tile_bytes, &raw_full[rs]);
             }
         }
     } else if (warp == 1) {
@@ -420,8 +440,9 @@ cudaError_t launch_a8(const void *layout, const Dims &d, const int8_t *x8, int64
     p.layout = (const uint8_t *)layout; p.dx = dx; p.y = y; p.status = status; p.d = d; p.M = (int)M;
     p.partial = partial; p.counters = counters; p.f16 = act_f16;
     p.raw_stage_bytes = (d.tile_bytes + 1023) / 1024 * 1024;
-    const size_t smem = (size_t)A8_STAGES * (A8_A_STAGE_BYTES + BN * 128) + (size_t)A8_RAW_STAGES * p.raw_stage_bytes +
-                        (size_t)8 * 2 * 16 * carrier_table_stride(B) + (size_t)A8_SRING * 128 * GPT * 4 + 512 + 256;
+    static_assert(A8_STAGES == 2 && A8_A_STAGE_BYTES == 128 * 128 && A8_SRING == 8, "a8_fixed_smem spells these out");
+    if (p.raw_stage_bytes != a8_raw_stage_bytes(B, G)) return cudaErrorInvalidConfiguration;
+    const size_t smem = (size_t)a8_fixed_smem(B, G, BN) + (size_t)a8_raw_stages(B, G, BN) * p.raw_stage_bytes;
     auto kern = gemm_a8_kernel<B, G, BN>;
     static std::atomic<uint64_t> attr_done{0};   // per kernel instantiation: the devices it has been set on
     cudaError_t ea = ensure_func_attr(kern, attr_done, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);

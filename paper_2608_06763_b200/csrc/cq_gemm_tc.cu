@@ -3,8 +3,9 @@
 // right before tcgen05.mma consumes them; accumulators live in TMEM.
 //
 // Roles inside a CTA (output tiles of 128 channels x BN or 2 BN tokens):
-//   warp 0      producer: bulk-copies raw layout tiles (codes + co-located group parameters) and
-//               TMA-loads activation tiles x[BN x 64] (128-byte swizzle) into a ring of stages
+//   warp 0      TMA-loads activation tiles x[BN x 64] (128-byte swizzle) into a ring of stages; nothing but the wait
+//               for a stage stands between the MMAs that free it and the copy that refills it
+//   warp 18     bulk-copies raw layout tiles (codes + co-located group parameters) into their own ring (2-4 deep)
 //   warp 1      allocates TMEM, issues tcgen05.mma (one elected lane), commits to mbarriers
 //   warps 2..17 decode: raw tile -> s_g * q(|k|/M) * sign (Eq. cubic; q by the half2 Horner form of
 //               Eq. gpu-horner on the power-of-two-normalised code, scale in fp32), rounded to bf16 and stored in

@@ -15,9 +15,8 @@ namespace {
 using namespace tc;
 
 constexpr int DEC_WARPS = 16;                 // decoder / epilogue warps
-constexpr int TC_THREADS = 64 + 32 * DEC_WARPS;
+constexpr int TC_THREADS = 64 + 32 * DEC_WARPS + 32;   // producer of activations, MMA issuer, decoders, producer of raw tiles
 constexpr int A_STAGE_BYTES = 128 * 128;  // 128 rows x 64 bf16
-constexpr int RAW_STAGES = 2;
 
 // ---------------------------------------------------------------- decode helpers
 // Two reconstructed weights s * sign(k) * q(|k| / M) of one pair, rounded to bf16 (the dense path
@@ -95,6 +94,13 @@ struct TcParams {
 
 // ---------------------------------------------------------------- the kernel (model dtype)
 constexpr int tc_stages(int BN, int NACC) { return BN * NACC >= 512 ? 2 : (BN == 256 ? 3 : 4); }
+// Raw layout tiles in flight per CTA: as many as the shared memory left by the operand ring holds, two to four.
+constexpr int tc_raw_stage_bytes(int B, int G) { return (2048 * B + 1024 * (TILE / G) + 1023) / 1024 * 1024; }
+constexpr int tc_raw_stages(int B, int G, int BN, int NACC) {
+    const int left = 226 * 1024 - 512 - tc_stages(BN, NACC) * (A_STAGE_BYTES + NACC * BN * 128);
+    const int n = left / tc_raw_stage_bytes(B, G);
+    return n > 4 ? 4 : n < 2 ? 2 : n;
+}
 
 __device__ __forceinline__ void named_barrier_sync(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
@@ -150,6 +156,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
     constexpr int GPT = TILE / G;
     constexpr int STAGES = tc_stages(BN, NACC);        // ring of 64-wide k blocks
+    constexpr int RAW_STAGES = tc_raw_stages(B, G, BN, NACC);
     constexpr int B_TILE_BYTES = BN * 128;             // one TMA box: BN tokens x 64 k
     constexpr int B_STAGE_BYTES = NACC * B_TILE_BYTES;
     constexpr int BNT = BN * NACC;                     // tokens per tile
@@ -198,16 +205,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
     SegWalk<SK> walk(prm);
     Seg seg;
     if (warp == 0) {
-        // ===== producer
+        // ===== producer of the activation tiles.  Nothing but the wait for the stage stands between the MMAs
+        // that free it and the TMA that refills it: with two stages that latency is on the critical path.
         if (lane == 0) {
-            int kbc = 0, tcnt = 0;     // 64-wide k blocks and layout tiles issued so far (they index the rings)
+            int kbc = 0;     // 64-wide k blocks issued so far (they index the ring)
             while (walk.next(seg)) {
-                const uint8_t *tiles = prm.layout + (size_t)seg.nb * d.KT * (size_t)d.tile_bytes;
-                for (int t = seg.k0; t < seg.k1; ++t, ++tcnt) {
-                    const int rs = tcnt % RAW_STAGES;
-                    if (tcnt >= RAW_STAGES) wait(&raw_empty[rs], ((tcnt / RAW_STAGES) - 1) & 1, 1);
-                    mbar_arrive_expect_tx(&raw_full[rs], (uint32_t)d.tile_bytes);
-                    bulk_load(sRaw + rs * prm.raw_stage_bytes, tiles + (size_t)t * d.tile_bytes, (uint32_t)d.tile_bytes, &raw_full[rs]);
+                for (int t = seg.k0; t < seg.k1; ++t) {
                     for (int half_k = 0; half_k < 2; ++half_k, ++kbc) {
                         const int s = kbc % STAGES;
                         if (kbc >= STAGES) wait(&st_empty[s], ((kbc / STAGES) - 1) & 1, 2);
@@ -216,6 +219,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                         for (int a = 0; a < NACC; ++a)
                             tma_load_2d(sB + s * B_STAGE_BYTES + a * B_TILE_BYTES, &xmap, &b_full[s], (2 * t + half_k) * 64, seg.mt * BNT + a * BN);
                     }
+                }
+            }
+        }
+    } else if (warp == 2 + DEC_WARPS) {
+        // ===== producer of the raw layout tiles (its own warp, so that a wait for the decoders never delays
+        // an activation tile)
+        if (lane == 0) {
+            int tcnt = 0;    // layout tiles issued so far
+            while (walk.next(seg)) {
+                const uint8_t *tiles = prm.layout + (size_t)seg.nb * d.KT * (size_t)d.tile_bytes;
+                for (int t = seg.k0; t < seg.k1; ++t, ++tcnt) {
+                    const int rs = tcnt % RAW_STAGES;
+                    if (tcnt >= RAW_STAGES) wait(&raw_empty[rs], ((tcnt / RAW_STAGES) - 1) & 1, 1);
+                    mbar_arrive_expect_tx(&raw_full[rs], (uint32_t)d.tile_bytes);
+                    bulk_load(sRaw + rs * prm.raw_stage_bytes, tiles + (size_t)t * d.tile_bytes, (uint32_t)d.tile_bytes, &raw_full[rs]);
                 }
             }
         }
@@ -482,6 +500,8 @@ cudaError_t launch_bn(const void *layout, const Dims &d, const uint16_t *x, uint
     p.layout = (const uint8_t *)layout; p.y = y; p.status = status; p.d = d; p.M = (int)M;
     p.raw_stage_bytes = (d.tile_bytes + 1023) / 1024 * 1024;
     p.MT = plan.token_tiles; p.t_full = plan.t_full; p.p2 = plan.p2;
+    constexpr int RAW_STAGES = tc_raw_stages(B, G, BN, NACC);
+    if (p.raw_stage_bytes != tc_raw_stage_bytes(B, G)) return cudaErrorInvalidConfiguration;
     const size_t smem = (size_t)STAGES * (A_STAGE_BYTES + NACC * BN * 128) + (size_t)RAW_STAGES * p.raw_stage_bytes + 256;
     auto kern = gemm_tc_kernel<B, G, BN, NACC, SK>;
     static std::atomic<uint64_t> attr_done{0};   // per kernel instantiation: the devices it has been set on
