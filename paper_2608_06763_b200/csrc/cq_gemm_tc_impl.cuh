@@ -93,11 +93,23 @@ struct TcParams {
 };
 
 // ---------------------------------------------------------------- the kernel (model dtype)
+// Depth of the ring of activation tiles (64-wide k blocks) and of the ring of decoded weight tiles.  The 512-token
+// tile has room for two activation stages only (64 KB each); its weight stages are 16 KB, so four of them let
+// the decoders run two layout tiles ahead of the MMAs instead of in lockstep with them.
 constexpr int tc_stages(int BN, int NACC) { return BN * NACC >= 512 ? 2 : (BN == 256 ? 3 : 4); }
-// Raw layout tiles in flight per CTA: as many as the shared memory left by the operand ring holds, two to four.
 constexpr int tc_raw_stage_bytes(int B, int G) { return (2048 * B + 1024 * (TILE / G) + 1023) / 1024 * 1024; }
+// Weight stages: up to four, fewer where the activation ring and two raw tiles leave less room.
+constexpr int tc_stages_a(int B, int G, int BN, int NACC) {
+    const int left = 226 * 1024 - 512 - tc_stages(BN, NACC) * NACC * BN * 128 - 2 * tc_raw_stage_bytes(B, G);
+    const int n = left / A_STAGE_BYTES;
+    return n > 4 ? 4 : n < 2 ? 2 : n;
+}
+constexpr int tc_ring_bytes(int B, int G, int BN, int NACC) {
+    return tc_stages_a(B, G, BN, NACC) * A_STAGE_BYTES + tc_stages(BN, NACC) * NACC * BN * 128;
+}
+// Raw layout tiles in flight per CTA: as many as the shared memory left by the operand rings holds, two to four.
 constexpr int tc_raw_stages(int B, int G, int BN, int NACC) {
-    const int left = 226 * 1024 - 512 - tc_stages(BN, NACC) * (A_STAGE_BYTES + NACC * BN * 128);
+    const int left = 226 * 1024 - 512 - tc_ring_bytes(B, G, BN, NACC);
     const int n = left / tc_raw_stage_bytes(B, G);
     return n > 4 ? 4 : n < 2 ? 2 : n;
 }
@@ -155,19 +167,20 @@ template <int B, int G, int BN, int NACC, bool SK>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
     constexpr int GPT = TILE / G;
-    constexpr int STAGES = tc_stages(BN, NACC);        // ring of 64-wide k blocks
+    constexpr int STAGES = tc_stages(BN, NACC);        // ring of activation tiles (64-wide k blocks)
+    constexpr int STAGES_A = tc_stages_a(B, G, BN, NACC);   // ring of decoded weight tiles
     constexpr int RAW_STAGES = tc_raw_stages(B, G, BN, NACC);
     constexpr int B_TILE_BYTES = BN * 128;             // one TMA box: BN tokens x 64 k
     constexpr int B_STAGE_BYTES = NACC * B_TILE_BYTES;
     constexpr int BNT = BN * NACC;                     // tokens per tile
     constexpr uint32_t TMEM_COLS = BNT < 32 ? 32 : BNT;
     extern __shared__ __align__(1024) uint8_t smem[];  // 1024-byte alignment is what the swizzled tiles need
-    uint8_t *sA = smem;                                        // STAGES x 16 KB
-    uint8_t *sB = sA + STAGES * A_STAGE_BYTES;                 // STAGES x BN x 128 B
+    uint8_t *sA = smem;                                        // STAGES_A x 16 KB
+    uint8_t *sB = sA + STAGES_A * A_STAGE_BYTES;               // STAGES x NACC x BN x 128 B
     uint8_t *sRaw = sB + STAGES * B_STAGE_BYTES;               // RAW_STAGES x raw_stage_bytes
     uint64_t *bars = reinterpret_cast<uint64_t *>(sRaw + RAW_STAGES * prm.raw_stage_bytes);
-    uint64_t *a_full = bars, *b_full = bars + STAGES, *st_empty = bars + 2 * STAGES;
-    uint64_t *raw_full = bars + 3 * STAGES, *raw_empty = raw_full + RAW_STAGES, *acc_full = raw_empty + RAW_STAGES;
+    uint64_t *a_full = bars, *a_empty = a_full + STAGES_A, *b_full = a_empty + STAGES_A, *b_empty = b_full + STAGES;
+    uint64_t *raw_full = b_empty + STAGES, *raw_empty = raw_full + RAW_STAGES, *acc_full = raw_empty + RAW_STAGES;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
     volatile int *s_last_p = reinterpret_cast<volatile int *>(tmem_slot + 1);    // "this CTA completes the tile"
     volatile int *gave_up = reinterpret_cast<volatile int *>(tmem_slot + 2);     // a bounded wait ran out somewhere in the CTA
@@ -180,7 +193,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
         return;
     }
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&a_full[s], DEC_WARPS); mbar_init(&b_full[s], 1); mbar_init(&st_empty[s], 1); }
+        for (int s = 0; s < STAGES_A; ++s) { mbar_init(&a_full[s], DEC_WARPS); mbar_init(&a_empty[s], 1); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1); }
         for (int s = 0; s < RAW_STAGES; ++s) { mbar_init(&raw_full[s], 1); mbar_init(&raw_empty[s], DEC_WARPS); }
         mbar_init(acc_full, 1);
         fence_barrier_init();
@@ -213,7 +227,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                 for (int t = seg.k0; t < seg.k1; ++t) {
                     for (int half_k = 0; half_k < 2; ++half_k, ++kbc) {
                         const int s = kbc % STAGES;
-                        if (kbc >= STAGES) wait(&st_empty[s], ((kbc / STAGES) - 1) & 1, 2);
+                        if (kbc >= STAGES) wait(&b_empty[s], ((kbc / STAGES) - 1) & 1, 2);
                         mbar_arrive_expect_tx(&b_full[s], B_STAGE_BYTES);
 #pragma unroll
                         for (int a = 0; a < NACC; ++a)
@@ -245,12 +259,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
             while (walk.next(seg)) {
                 const int nkb = 2 * (seg.k1 - seg.k0);
                 for (int i = 0; i < nkb; ++i, ++kbc) {
-                    const int s = kbc % STAGES;
-                    const uint32_t ph = (kbc / STAGES) & 1;
-                    wait(&a_full[s], ph, 3);
-                    wait(&b_full[s], ph, 4);
+                    const int s = kbc % STAGES, sa = kbc % STAGES_A;
+                    wait(&a_full[sa], (kbc / STAGES_A) & 1, 3);
+                    wait(&b_full[s], (kbc / STAGES) & 1, 4);
                     tc_fence_after();
-                    const uint64_t adesc = smem_desc_sw128(smem_u32(sA + s * A_STAGE_BYTES));
+                    const uint64_t adesc = smem_desc_sw128(smem_u32(sA + sa * A_STAGE_BYTES));
 #pragma unroll
                     for (int a = 0; a < NACC; ++a) {
                         const uint64_t bdesc = smem_desc_sw128(smem_u32(sB + s * B_STAGE_BYTES + a * B_TILE_BYTES));
@@ -258,7 +271,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                         for (int k = 0; k < 4; ++k)  // four K = 16 steps, 32 bytes apart inside the swizzle atom
                             umma_bf16(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, (i | k) != 0);
                     }
-                    umma_commit(&st_empty[s]);  // frees the stage when these MMAs have read it
+                    umma_commit(&a_empty[sa]);  // frees the two stages when these MMAs have read them
+                    umma_commit(&b_empty[s]);
                 }
                 // The accumulators of this segment are complete when these MMAs are.  The next segment's first MMA
                 // overwrites them, but it waits for a decoded stage, and the decoders decode again only after
@@ -310,8 +324,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
             }
 #pragma unroll 1
             for (int half_k = 0; half_k < 2; ++half_k) {
-                const int kb = kbc++, s = kb % STAGES;
-                if (kb >= STAGES) wait(&st_empty[s], ((kb / STAGES) - 1) & 1, 6);
+                const int kb = kbc++, s = kb % STAGES_A;
+                if (kb >= STAGES_A) wait(&a_empty[s], ((kb / STAGES_A) - 1) & 1, 6);
                 uint8_t *a_stage = sA + s * A_STAGE_BYTES;
                 // rows g (low) and g + 8 (high) of the row block: their 128-byte rows in the stage
                 uint8_t *row_lo = a_stage + (rb * 2 + 0) * 1024 + g * 128;
@@ -493,7 +507,6 @@ cudaError_t launch_bn(const void *layout, const Dims &d, const uint16_t *x, uint
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
-    constexpr int STAGES = tc_stages(BN, NACC);
     const TcPlan plan = gemm_tc_plan(d, M);
     if (plan.bnt != BN * NACC || (plan.p2 > 0) != SK) return cudaErrorInvalidConfiguration;
     TcParams p;
@@ -502,7 +515,8 @@ cudaError_t launch_bn(const void *layout, const Dims &d, const uint16_t *x, uint
     p.MT = plan.token_tiles; p.t_full = plan.t_full; p.p2 = plan.p2;
     constexpr int RAW_STAGES = tc_raw_stages(B, G, BN, NACC);
     if (p.raw_stage_bytes != tc_raw_stage_bytes(B, G)) return cudaErrorInvalidConfiguration;
-    const size_t smem = (size_t)STAGES * (A_STAGE_BYTES + NACC * BN * 128) + (size_t)RAW_STAGES * p.raw_stage_bytes + 256;
+    const size_t smem = (size_t)tc_ring_bytes(B, G, BN, NACC) + (size_t)RAW_STAGES * p.raw_stage_bytes + 256;
+    static_assert(tc_ring_bytes(B, G, BN, NACC) + tc_raw_stages(B, G, BN, NACC) * tc_raw_stage_bytes(B, G) + 256 <= 227 * 1024, "shared memory");
     auto kern = gemm_tc_kernel<B, G, BN, NACC, SK>;
     static std::atomic<uint64_t> attr_done{0};   // per kernel instantiation: the devices it has been set on
     cudaError_t ea = ensure_func_attr(kern, attr_done, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
