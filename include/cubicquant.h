@@ -66,7 +66,10 @@ double cq_effective_bits(int B, int G);
  * padding of N and K up to multiples of 128).  0 if the arguments are unsupported. */
 size_t cq_layout_bytes(int B, int G, int64_t N, int64_t K);
 /* Bytes of scratch cq_gemm needs for this problem (split-K partial sums and arrival counters;
- * Dynamic A8 adds the INT8 activation carrier and its row scales).  Never 0 for valid input. */
+ * Dynamic A8 adds the INT8 activation carrier and its row scales).  Never 0 for valid input.  The split-K
+ * schedule, and with it this size, depends on the number of multiprocessors of the current device (148 are
+ * assumed when no device can be asked): ask with the device current on which cq_gemm will run; cq_gemm
+ * checks workspace_bytes against the device it runs on and returns CQ_ERR_WORKSPACE if it is too small. */
 size_t cq_workspace_bytes(int B, int G, int64_t M, int64_t N, int64_t K, int mode);
 /* Zero the arrival counters of a workspace.  Call once after allocating it (and after any
  * cq_gemm that returned an error); cq_gemm leaves the counters zero when it completes. */
