@@ -393,7 +393,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
             const int q4 = warp & 3;                       // TMEM lane quarter this warp may access
             const int cp = dw >> 2;                        // which of four column parts
             const int64_t n = (int64_t)seg.nb * TILE + q4 * 32 + lane;
-            if (whole) {
+            if ((d.N & 7) == 0 && (!SK || (int64_t)blockIdx.x < prm.t_full)) {
+                // A CTA whose only work is this whole tile, and rows of y that start on 16-byte boundaries: the tile goes
+                // through shared memory (the activation ring is idle by now: every MMA has completed and nothing more is
+                // loaded; a CTA with a run of several segments may already be loading the next one) as
+                // [token][128 channels] in the output dtype, and leaves it in 16-byte pieces, eight channels of one
+                // token per thread, instead of one 2-byte store per output.
+                uint16_t *stage = reinterpret_cast<uint16_t *>(sB);
+#pragma unroll 1
+                for (int c0 = cp * 32; c0 < BNT; c0 += 128) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)c0, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) stage[(c0 + i) * TILE + q4 * 32 + lane] = float_to_act(__uint_as_float(r[i]), prm.f16);
+                }
+                named_barrier_sync(1, 32 * DEC_WARPS);
+                const int64_t m0 = (int64_t)seg.mt * BNT, n0 = (int64_t)seg.nb * TILE;
+                for (int c = dec_tid; c < BNT * (TILE / 8); c += 32 * DEC_WARPS) {
+                    const int tok = c / (TILE / 8), part = c % (TILE / 8);
+                    if (m0 + tok < prm.M && n0 + part * 8 < d.N)   // N is a multiple of 8: a piece is inside or outside as a whole
+                        *reinterpret_cast<uint4 *>(prm.y + (m0 + tok) * d.N + n0 + part * 8) = *reinterpret_cast<const uint4 *>(stage + tok * TILE + part * 8);
+                }
+            } else if (whole) {
 #pragma unroll 1
                 for (int c0 = cp * 32; c0 < BNT; c0 += 128) {
                     uint32_t r[32];
