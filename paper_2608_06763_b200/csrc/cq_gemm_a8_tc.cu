@@ -356,22 +356,27 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
                 const int e_z = (int)*reinterpret_cast<volatile uint32_t *>(tmem_slot + 5);
                 const int e_tile = (int)*reinterpret_cast<volatile uint32_t *>(tmem_slot + 6);
                 float *pslot = prm.partial + ((size_t)(e_tile - prm.t_full) * prm.slices + e_z) * (size_t)(BN * TILE) + drow;
-                auto store_all = [&](auto f16c) {
-                    constexpr bool F16 = decltype(f16c)::value;
+                auto store_all = [&](auto f16c, auto stagedc) {
+                    constexpr bool F16 = decltype(f16c)::value, STAGED = decltype(stagedc)::value;
 #pragma unroll
                     for (int i = 0; i < QCOLS; ++i) {
                         const int64_t m = (int64_t)e_mt * BN + cq4 * QCOLS + i;
                         if (m < prm.M) {
                             if (e_nz == 1) {
                                 const float v = acc[i] * (prm.dx[m] * (1.0f / 127.0f));
-                                prm.y[m * d.N + n] = float_to_act(v, F16);
+                                if constexpr (STAGED) reinterpret_cast<uint16_t *>(sB)[(cq4 * QCOLS + i) * TILE + drow] = float_to_act(v, F16);
+                                else prm.y[m * d.N + n] = float_to_act(v, F16);
                             } else {
                                 pslot[(size_t)(cq4 * QCOLS + i) * TILE] = acc[i];
                             }
                         }
                     }
                 };
-                if (*reinterpret_cast<volatile uint32_t *>(tmem_slot + 3)) store_all(std::true_type{}); else store_all(std::false_type{});
+                // A whole tile whose rows of y start on 16-byte boundaries goes through shared memory (the activation
+                // ring is idle: every MMA has completed) and is copied out in 16-byte pieces after the CTA's barrier.
+                const bool f16o = *reinterpret_cast<volatile uint32_t *>(tmem_slot + 3) != 0;
+                if (e_nz == 1 && (d.N & 7) == 0) { if (f16o) store_all(std::true_type{}, std::true_type{}); else store_all(std::false_type{}, std::true_type{}); }
+                else { if (f16o) store_all(std::true_type{}, std::false_type{}); else store_all(std::false_type{}, std::false_type{}); }
             }
         }
     }
@@ -382,6 +387,17 @@ gemm_a8_kernel(const __grid_constant__ CUtensorMap xmap, A8Params prm) {
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+    if (*reinterpret_cast<volatile uint32_t *>(tmem_slot + 4) == 1 && (d.N & 7) == 0 && !*reinterpret_cast<volatile uint32_t *>(tmem_slot + 2)) {
+        // the staged tile [token][128 channels]: eight channels of one token per thread and step
+        const int64_t m0 = (int64_t)*reinterpret_cast<volatile uint32_t *>(tmem_slot + 8) * BN;
+        const int64_t n0 = (int64_t)*reinterpret_cast<volatile uint32_t *>(tmem_slot + 7) * TILE;
+        const uint16_t *stage = reinterpret_cast<const uint16_t *>(sB);
+        for (int c = threadIdx.x; c < BN * (TILE / 8); c += A8_THREADS) {
+            const int tok = c / (TILE / 8), part = c % (TILE / 8);
+            if (m0 + tok < prm.M && n0 + part * 8 < d.N)
+                *reinterpret_cast<uint4 *>(prm.y + (m0 + tok) * d.N + n0 + part * 8) = *reinterpret_cast<const uint4 *>(stage + tok * TILE + part * 8);
+        }
+    }
     if (*reinterpret_cast<volatile uint32_t *>(tmem_slot + 4) > 1) {
         // The last CTA of this output tile to arrive adds the slices in K order and applies d_x / 127.  The barrier
         // above ordered the CTA's partial stores before thread 0's release.  (Tile, slice count and position are read
