@@ -205,13 +205,13 @@ int cq_debug_a8_partials(const void *layout, int B, int G, const int8_t *x8, int
  * workspace: device pointer, 16-byte aligned, at least 512 bytes. */
 int cq_debug_wait_timeout(void *workspace, size_t workspace_bytes, int64_t limit_cycles, void *stream);
 
-/* How cq_gemm(..., CQ_MODEL_DTYPE, ...) with M > 16 spreads this problem over the current device (host-side
- * query, launches nothing; the paper has no counterpart).  plan must hold five values: plan[0] = tokens per output
- * tile, plan[1] = CTAs that compute one whole 128-channel x plan[0]-token tile each, plan[2] = CTAs that share the
- * remaining tiles, each taking a contiguous run of (tile, K) units (stream-K; 0 when every tile is computed whole),
- * plan[3] = those remaining tiles, plan[4] = 1 when a run may cross from one tile into the next, 0 when every
- * shared tile is cut into the same number of runs.  CQ_ERR_INVALID_ARG for M <= 16 or a null pointer. */
-int cq_debug_gemm_plan(int B, int G, int64_t M, int64_t N, int64_t K, int64_t *plan);
+/* How cq_gemm(..., mode, ...) with M > 16 spreads this problem over the current device (host-side query, launches
+ * nothing; the paper has no counterpart).  plan must hold five values: plan[0] = tokens per output tile, plan[1] =
+ * CTAs that compute one whole 128-channel x plan[0]-token tile each, plan[2] = CTAs that share the remaining tiles,
+ * each taking a contiguous run of (tile, K) units (0 when every tile is computed whole), plan[3] = those remaining
+ * tiles, plan[4] = 1 when a run may cross from one tile into the next, 0 when every shared tile is cut into the same
+ * number of runs (always 0 in CQ_DYN_A8).  CQ_ERR_INVALID_ARG for M <= 16, an unknown mode or a null pointer. */
+int cq_debug_gemm_plan(int B, int G, int64_t M, int64_t N, int64_t K, int mode, int64_t *plan);
 
 /* ---- Offline encoder (the step before the hot path; Sections 4.1 and 4.3) --------------------------
  * W[N][K] float, logical signed codes k[N][K] int8 (what cq_pack_codes takes), scale[N][K/G] float,

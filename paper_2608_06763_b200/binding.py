@@ -69,7 +69,7 @@ def lib():
         L.cq_decode_carriers.argtypes = [vp, i, i, i64, i64, vp, vp]
         L.cq_decode_weights.argtypes = [vp, i, i, i64, i64, vp, vp]
         L.cq_debug_a8_partials.argtypes = [vp, i, i, vp, i64, i64, i64, vp, vp]
-        L.cq_debug_gemm_plan.argtypes = [i, i, i64, i64, i64, vp]
+        L.cq_debug_gemm_plan.argtypes = [i, i, i64, i64, i64, i, vp]
         L.cq_debug_gemm_plan.restype = i
         L.cq_debug_wait_timeout.argtypes = [vp, sz, i64, vp]
         L.cq_debug_wait_timeout.restype = i
@@ -290,10 +290,10 @@ def cq_debug_a8_partials(pw: PackedWeights, x8: torch.Tensor) -> torch.Tensor:
     return out
 
 
-def cq_debug_gemm_plan(B: int, G: int, M: int, N: int, K: int) -> dict:
-    """How the model-dtype GEMM (M > 16) spreads a problem over the current device."""
+def cq_debug_gemm_plan(B: int, G: int, M: int, N: int, K: int, mode: int = CQ_MODEL_DTYPE) -> dict:
+    """How the large-M GEMM of `mode` (M > 16) spreads a problem over the current device."""
     out = (C.c_int64 * 5)()
-    _check(lib().cq_debug_gemm_plan(B, G, M, N, K, out), "cq_debug_gemm_plan")
+    _check(lib().cq_debug_gemm_plan(B, G, M, N, K, mode, out), "cq_debug_gemm_plan")
     return {"token_tile": out[0], "whole_tile_ctas": out[1], "stream_k_ctas": out[2], "stream_k_tiles": out[3],
             "runs_cross_tiles": bool(out[4])}
 

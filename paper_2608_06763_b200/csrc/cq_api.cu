@@ -388,14 +388,20 @@ int cq_decode_weights(const void *layout, int B, int G, int64_t N, int64_t K, fl
     return wrap(launch_decode_weights(layout, d, What, (cudaStream_t)stream));
 }
 
-int cq_debug_gemm_plan(int B, int G, int64_t M, int64_t N, int64_t K, int64_t *plan) {
-    if (!plan || M <= 16) return CQ_ERR_INVALID_ARG;
+int cq_debug_gemm_plan(int B, int G, int64_t M, int64_t N, int64_t K, int mode, int64_t *plan) {
+    if (!plan || M <= 16 || (mode != CQ_MODEL_DTYPE && mode != CQ_DYN_A8)) return CQ_ERR_INVALID_ARG;
     const int st = check_format(B, G, N, K);
     if (st != CQ_OK) return st;
     const Dims d = make_dims(B, G, N, K);
-    const TcPlan tp = gemm_tc_plan(d, M);
-    plan[0] = tp.bnt; plan[1] = tp.t_full; plan[2] = tp.p2; plan[3] = (int64_t)d.NB * tp.token_tiles - tp.t_full;
-    plan[4] = tp.crossing;
+    if (mode == CQ_MODEL_DTYPE) {
+        const TcPlan tp = gemm_tc_plan(d, M);
+        plan[0] = tp.bnt; plan[1] = tp.t_full; plan[2] = tp.p2; plan[3] = (int64_t)d.NB * tp.token_tiles - tp.t_full;
+        plan[4] = tp.crossing;
+    } else {
+        const A8Plan ap = gemm_a8_plan(d, M);
+        const int64_t shared = (int64_t)d.NB * ap.token_tiles - ap.t_full;
+        plan[0] = ap.bn; plan[1] = ap.t_full; plan[2] = shared * ap.slices; plan[3] = shared; plan[4] = 0;
+    }
     return CQ_OK;
 }
 

@@ -69,12 +69,13 @@ def test_gemm_plan_shares_the_last_round_only_when_it_pays():
     L = cq.lib()
     plan = (ctypes.c_int64 * 5)()
 
-    def ask(B, G, M, N, K):
-        assert L.cq_debug_gemm_plan(B, G, M, N, K, plan) == 0
+    def ask(B, G, M, N, K, mode=0):
+        assert L.cq_debug_gemm_plan(B, G, M, N, K, mode, plan) == 0
         return list(plan)
 
-    assert L.cq_debug_gemm_plan(4, 128, 16, 4096, 4096, plan) == -1       # M <= 16 is the small-M kernel's
-    assert L.cq_debug_gemm_plan(4, 128, 64, 4096, 4096, None) == -1
+    assert L.cq_debug_gemm_plan(4, 128, 16, 4096, 4096, 0, plan) == -1    # M <= 16 is the small-M kernel's
+    assert L.cq_debug_gemm_plan(4, 128, 64, 4096, 4096, 0, None) == -1
+    assert L.cq_debug_gemm_plan(4, 128, 64, 4096, 4096, 7, plan) == -1
     for (M, N, K) in [(1024, 28672, 4096), (1024, 4096, 14336), (4096, 8192, 28672), (40, 256, 8192), (33, 100, 4224),
                       (4096, 57344, 8192), (1024, 6144, 4096), (17, 128, 128), (300, 200, 1024), (32, 28672, 4096)]:
         bnt, whole, runs, shared, crossing = ask(4, 128, M, N, K)
@@ -90,3 +91,8 @@ def test_gemm_plan_shares_the_last_round_only_when_it_pays():
     assert ask(4, 128, 1024, 28672, 4096) == [512, 444, 32, 4, 0]     # three whole rounds, four tiles cut into eight runs each
     assert ask(4, 128, 4096, 57344, 8192)[2] == 0                     # 24 rounds and a bit: sharing would not pay
     assert ask(4, 128, 17, 128, 128)[2] == 0                          # one layout tile of K cannot be cut
+    # Dynamic A8: 256-token tiles at G = 128; only the tiles of the last round are cut, into equal slices
+    assert ask(4, 128, 1024, 6144, 4096, 1) == [256, 148, 132, 44, 0]
+    assert ask(4, 128, 300, 200, 512, 1)[2] == 0                      # four blocks of K: nothing to cut
+    bn, whole, runs, shared, crossing = ask(4, 128, 100, 200, 2048, 1)
+    assert (bn, whole, shared, crossing) == (128, 0, 2, 0) and runs in (4, 6, 8)

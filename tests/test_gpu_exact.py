@@ -97,8 +97,10 @@ def test_a8_small_m_kernel_bit_exact(B, G, M):
 @pytest.mark.parametrize("G", [32, 64, 128])
 @pytest.mark.parametrize("B", [1, 2, 3, 4, 5, 6, 7, 8])
 def test_a8_tcgen05_kernel_bit_exact(B, G, M, K):
-    # K = 2048 with few output tiles cuts K into slices (split-K); M = 300 runs without
+    # K = 2048 with few output tiles cuts K into slices (the last CTA of a tile adds them); K = 512 runs without
     N = 200
+    plan = cq.cq_debug_gemm_plan(B, G, M, N, K, cq.CQ_DYN_A8)
+    assert (plan["stream_k_ctas"] > plan["stream_k_tiles"]) == (K == 2048), plan
     nnz = 8 if K == 512 else 2
     c = edge_case(N, K, B, G, seed=530 + B, scales=power_of_two_scales(N * (K // G), 540 + B, 1 if K == 512 else 0))
     a8_exact(c, integer_activations(M, K, G, nnz, seed=550 + M))

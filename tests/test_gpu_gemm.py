@@ -194,6 +194,8 @@ def test_a8_gemm_token_tiles_and_split_k(M, G):
     # capped by the group count) and cuts K into slices combined in slice order; two calls on one
     # workspace must agree bit for bit (arrival counters are left cleared)
     N, K, B = 200, 2048, 4
+    plan = cq.cq_debug_gemm_plan(B, G, M, N, K, cq.CQ_DYN_A8)
+    assert plan["stream_k_ctas"] > plan["stream_k_tiles"] > 0, plan     # the tiles are cut into slices
     c = logical_case(N, K, B, G, seed=190 + M)
     c.k[7, 100:140] = -(1 << (B - 1))
     c = Case(c.k, c.s, c.a, c.b, B, G)
