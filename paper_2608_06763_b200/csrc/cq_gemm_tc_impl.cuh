@@ -322,8 +322,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                 tc_lo = make_coef<B>(q_lo); tc_hi = make_coef<B>(q_hi);
                 tfix = B > 1 && __any_sync(0xffffffffu, (q_lo.x | q_hi.x) >> 31);
             }
-#pragma unroll 1
-            for (int half_k = 0; half_k < 2; ++half_k) {
+            // one 64-wide block: this warp's unit JQ of the tile (unit = two 16-wide chunks of 16 rows)
+            auto do_block = [&](auto jq_block) {
                 const int kb = kbc++, s = kb % STAGES_A;
                 if (kb >= STAGES_A) wait(&a_empty[s], ((kb / STAGES_A) - 1) & 1, 6);
                 uint8_t *a_stage = sA + s * A_STAGE_BYTES;
@@ -371,16 +371,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap xmap, TcParams prm) {
                     if (!prm.f16) { if (!fix) emit(std::false_type{}, std::false_type{}); else emit(std::true_type{}, std::false_type{}); }
                     else { if (!fix) emit(std::false_type{}, std::true_type{}); else emit(std::true_type{}, std::true_type{}); }
                 };
-                switch (half_k * 2 + jh) {
-                    case 0: do_unit(std::integral_constant<int, 0>{}); break;
-                    case 1: do_unit(std::integral_constant<int, 1>{}); break;
-                    case 2: do_unit(std::integral_constant<int, 2>{}); break;
-                    default: do_unit(std::integral_constant<int, 3>{}); break;
-                }
+                do_unit(jq_block);
                 fence_proxy_async();   // generic-proxy stores -> visible to the tensor core's async proxy
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&a_full[s]);
-            }
+            };
+            // the first 64-wide block of the tile holds units 0 and 1, the second units 2 and 3; jh picks the warp's
+            if (jh == 0) { do_block(std::integral_constant<int, 0>{}); do_block(std::integral_constant<int, 2>{}); }
+            else { do_block(std::integral_constant<int, 1>{}); do_block(std::integral_constant<int, 3>{}); }
             __syncwarp();
             if (lane == 0) mbar_arrive(&raw_empty[rs]);
         }
