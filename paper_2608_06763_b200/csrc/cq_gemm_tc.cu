@@ -36,7 +36,7 @@ int gemm_tc_token_tile(int64_t M) { return M <= 32 ? 32 : M <= 64 ? 64 : M <= 12
 //       length + 4 .. 10 (the fill, the partial tile's trip through L2 and, for one CTA per tile, the addition
 //       of the partial tiles; the more the wider the token tile), and r s runs take ceil(r s / SMs) rounds;
 //   (a) one run per SM, cut anywhere: the best balance, but most runs cross from one tile into the next (two
-//       fills, two partial tiles: length + 6 .. 16).
+//       fills, two partial tiles: length + 10 .. 22; recalibrated against forced plans at M = 64 .. 4096).
 // The kernel that can share tiles runs about 5 % slower on every tile of the launch than the one that cannot
 // (measured at M = 4096, N = 57344, K = 8192, and at M = 1024, N = 6144, K = 4096; merely compiling the partial-tile
 // code into the kernel costs that much), so it is a separate instantiation and sharing has to save more.
@@ -61,7 +61,7 @@ TcPlan gemm_tc_plan(const Dims &d, int64_t M) {
         int64_t pa = sms;
         if (pa > V2 / 4) pa = V2 / 4;               // at least four layout tiles per run
         if (pa > r) {
-            const double c = (double)V2 / (double)pa + 6.0 + 10.0 * wide;
+            const double c = (double)V2 / (double)pa + 10.0 + 12.0 * wide;
             if (c < best) { best = c; best_p2 = pa; best_crossing = 1; }
         }
         if (best_p2 > 0 && (whole - best) / all > 0.06) { p.p2 = (int)best_p2; p.crossing = best_crossing; p.t_full = T - r; }

@@ -130,7 +130,7 @@ def test_tensor_core_gemm_wide_token_tile(M):
 # tile; a last round of 76 tiles shared by one run per SM, so that runs cross from one tile into the next (the
 # kernel of cq_gemm_tc_sk.cu).
 STREAM_K_SHAPES = [(256, 8192, 40, False), (100, 4096 + 128, 33, False), (128 * 150, 4096, 40, False),
-                   (384, 8192, 700, False), (128 * (148 + 76), 2048, 20, True)]
+                   (384, 8192, 700, False), (128 * (148 + 76), 4096, 20, True)]
 
 
 @pytest.mark.parametrize("act", ["bf16", "f16"])
